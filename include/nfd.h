@@ -1,0 +1,191 @@
+/*
+ * nfd.h -- C ABI of libnfd: the few-step denoising forward pass of a block-wise
+ * causal diffusion transformer with a frame-paged KV cache and k-frame
+ * speculative decoding (Next-Frame Diffusion, arxiv 2506.01380), for one
+ * NVIDIA B200 (sm_100a).
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers, "host" pointers ordinary host
+ *     memory.  The caller owns every pointer it passes.  The library owns the
+ *     context, its repacked weights, the KV cache, activations and graphs.
+ *   - All device work is enqueued on the CUDA stream given to nfd_create.
+ *     Calls are asynchronous with respect to the host unless stated otherwise.
+ *   - Every function returns 0 on success or a negative NFD_E_* code.  A failed
+ *     call leaves the cache and its counters unchanged.  Nothing throws or
+ *     aborts across this boundary.
+ *   - A frame is a latent [C, H, W] (row-major, fp32).  It is cut into
+ *     (H/p)*(W/p) tokens in row-major order over (row, col); a token's patch
+ *     vector is ordered (channel, py, px).
+ *   - "stream" (int) below is a batch slot: an independent generation stream
+ *     with its own cache, 0 <= stream < cfg.n_streams.
+ *   - Frames are numbered 0,1,2,... per stream since the last nfd_reset.  A
+ *     frame f attends to frames max(0, f - W) .. f  (W = cfg.ctx_frames):
+ *     bidirectionally inside f, causally to the earlier ones.
+ */
+#ifndef NFD_H_
+#define NFD_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NFD_OK          0
+#define NFD_E_BADCFG   -1   /* inconsistent or unsupported configuration          */
+#define NFD_E_NULLPTR  -2   /* a required pointer is NULL                          */
+#define NFD_E_ALIGN    -3   /* a device pointer is not 16-byte aligned             */
+#define NFD_E_RANGE    -4   /* an index / count argument is out of range           */
+#define NFD_E_STATE    -5   /* call not allowed in the cache's current state       */
+#define NFD_E_NOMEM    -6   /* device or host allocation failed                    */
+#define NFD_E_CUDA     -7   /* a CUDA runtime call failed                          */
+#define NFD_E_TIMEOUT  -8   /* a bounded device-side wait gave up                  */
+#define NFD_E_DEVICE   -9   /* a device-side consistency check failed              */
+
+#define NFD_DTYPE_FP32 0    /* validation mode: fp32 storage and arithmetic        */
+#define NFD_DTYPE_BF16 1    /* bf16 operands / cache, fp32 accumulation & residual */
+
+#define NFD_MAX_PASS_FRAMES 32   /* frames one forward pass can carry (streams x k) */
+
+typedef struct nfd_ctx nfd_ctx;
+
+/* Model and cache configuration.  Architecture: Section 3.1 of the paper (DiT
+ * with block-wise causal attention, adaLN-zero conditioning on timestep +
+ * action, 3D rotary embedding); sampler constants: Section 4.1. */
+typedef struct {
+    int n_layers, d_model, n_heads, head_dim, d_mlp;   /* n_heads*head_dim == d_model; head_dim in {32,64,128} */
+    int latent_c, latent_h, latent_w, patch;            /* tokens/frame T = (h/p)*(w/p); patch vector P = c*p*p  */
+    int n_actions;                                      /* one categorical action per frame                      */
+    int ctx_frames;                                     /* W: earlier frames a frame attends to                  */
+    int max_spec;                                       /* k_max: frames decoded together, 1..8                  */
+    int n_streams;                                      /* independent batch slots                               */
+    int dtype;                                          /* NFD_DTYPE_*                                           */
+    int norm;                                           /* 0 LayerNorm (no affine), 1 RMSNorm                    */
+    int act;                                            /* 0 exact (erf) GELU                                    */
+    int rope_t, rope_h, rope_w;                         /* even, sum == head_dim (Section 3.1, 3D pos. emb.)     */
+    float rope_theta, norm_eps, t_scale;                /* t_scale multiplies the FM time before the sinusoid    */
+    float sigma_d;                                      /* TrigFlow data scale (Section 4.1)                     */
+    float t_ctx_trig;                                   /* TrigFlow time of the context-noise level (Sec. 4.3)   */
+    int n_steps;                                        /* sampling steps S (Section 4.1 "Sampling": 4)          */
+} nfd_cfg;
+
+/* Weights: dev pointers, each matrix row-major [in, out], element type given by
+ * cfg.dtype (float or bf16).  Per-layer arrays are host arrays of n_layers dev
+ * pointers.  nfd_create copies and repacks them; the caller may free its
+ * copies afterwards. */
+typedef struct {
+    const void *w_pe, *b_pe;                 /* [P,d], [d]      patch embedding                          */
+    const void *w_t1, *b_t1, *w_t2, *b_t2;   /* [256,d],[d],[d,d],[d]  timestep-embedding MLP (SiLU)     */
+    const void *a_emb;                       /* [n_actions,d]   action embedding (linear on one-hot)     */
+    const void *const *w_mod, *const *b_mod; /* [d,6d],[6d]     adaLN: shift,scale,gate (attn), same (mlp) */
+    const void *const *w_qkv, *const *b_qkv; /* [d,3d],[3d]     columns: q | k | v, each head-major      */
+    const void *const *w_o,   *const *b_o;   /* [d,d],[d]                                                */
+    const void *const *w_fc1, *const *b_fc1; /* [d,d_mlp],[d_mlp]                                        */
+    const void *const *w_fc2, *const *b_fc2; /* [d_mlp,d],[d]                                            */
+    const void *w_fmod, *b_fmod;             /* [d,2d],[2d]     final adaLN: shift, scale                */
+    const void *w_out, *b_out;               /* [d,P],[P]       velocity head                            */
+} nfd_weights;
+
+/* Create a context.  `cuda_stream` is a cudaStream_t (NULL = legacy default
+ * stream).  Validates cfg (NFD_E_BADCFG), copies/repacks the weights, allocates
+ * the cache: n_streams x n_layers x (W + k_max) frame pages of K and of V.
+ * Synchronises the stream before returning. */
+int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cuda_stream);
+int nfd_destroy(nfd_ctx *ctx);
+
+/* Empty one batch slot's cache and restart its frame numbering at 0. */
+int nfd_reset(nfd_ctx *ctx, int stream);
+
+/* One forward pass v_theta(x_t | cached frames, t, action) (Section 3.2, the
+ * argument of the Flow-Matching loss) over k frames decoded together: they
+ * follow the cached frames, share the FM time t and the action, and are
+ * block-causal among themselves (Section 4.2).  x_t: dev fp32 [k,C,H,W], the
+ * model input (already in Flow-Matching scale).  v_out: dev fp32 [k,C,H,W].
+ * The k frames' K/V are left in scratch pages after the cached frames; they are
+ * not counted by the cache until a commit.  1 <= k <= k_max. */
+int nfd_denoise_step(nfd_ctx *ctx, int stream, const float *x_t, int k, float t, int action, float *v_out);
+
+/* As nfd_denoise_step, but the k frames start `offset` frames after the cached
+ * ones and the scratch K/V that earlier calls left for those `offset` frames
+ * serve as context (offset + k <= k_max).  A joint k-frame pass equals k
+ * single-frame calls with offset = 0..k-1. */
+int nfd_denoise_step_at(nfd_ctx *ctx, int stream, int offset, const float *x_t, int k, float t, int action,
+                        float *v_out);
+
+/* The same pass for n batch slots at once (independent streams, one launch):
+ * streams[n] host, x_t dev [n,k,C,H,W], t[n] host, actions[n] host,
+ * v_out dev [n,k,C,H,W].  n*k <= NFD_MAX_PASS_FRAMES. */
+int nfd_denoise_step_batched(nfd_ctx *ctx, int n, const int *streams, const float *x_t, int k, const float *t,
+                             const int *actions, float *v_out);
+
+/* Append n clean frames to the cache (Appendix "KV caching": the K/V of the
+ * noisy versions of generated frames are computed once and reused).  Each frame
+ * is perturbed to the context-noise level, x' = cos(t_ctx) x0 + sin(t_ctx)
+ * sigma_d z (Section 4.3), fed at that constant timestep with the action that
+ * produced it, and its K/V written to the next pages.  x0 dev fp32 [n,C,H,W];
+ * actions host [n]; ctx_noise dev fp32 [n,C,H,W] or NULL (z = 0).
+ * Requires no tentative frames (NFD_E_STATE).  1 <= n <= k_max. */
+int nfd_commit_frame(nfd_ctx *ctx, int stream, const float *x0, int n, const int *actions, const float *ctx_noise);
+
+/* Generate k frames speculatively under `action` (Section 4.2): S sampling
+ * steps (Section 4.1 "Sampling": denoise, then re-noise to the next timestep)
+ * over the k frames decoded together, then append the k clean frames as
+ * TENTATIVE.  noise dev fp32 [S,k,C,H,W] (N(0,1): step 0 is the initial sample,
+ * step s>0 the re-noising draw); ctx_noise dev [k,C,H,W] or NULL; x0_out dev
+ * fp32 [k,C,H,W] receives the clean frames.  Requires no tentative frames. */
+int nfd_speculate(nfd_ctx *ctx, int stream, int k, int action, const float *noise, const float *ctx_noise,
+                  float *x0_out);
+
+/* nfd_speculate for n batch slots at once: streams[n], actions[n] host;
+ * noise dev [S,n,k,C,H,W]; ctx_noise dev [n,k,C,H,W] or NULL; x0_out dev [n,k,C,H,W]. */
+int nfd_speculate_batched(nfd_ctx *ctx, int n, const int *streams, int k, const int *actions, const float *noise,
+                          const float *ctx_noise, float *x0_out);
+
+/* Resolve a speculation (Section 4.2: frames after the first action mismatch are
+ * discarded, generation resumes from the last verified frame): the first
+ * n_accept tentative frames become committed, the rest are dropped.  Counters
+ * only; no data moves.  0 <= n_accept <= n_tentative. */
+int nfd_rollback(nfd_ctx *ctx, int stream, int n_accept);
+
+/* Cache counters (host ints, any may be NULL): committed frames, tentative
+ * frames, and the first frame the next new frame can see. */
+int nfd_kv_state(nfd_ctx *ctx, int stream, int *n_committed, int *n_tentative, int *window_first);
+
+/* 64-bit digest of the counters and of the raw K/V bits of the visible cached
+ * frames (the last W), in frame order.  Synchronises the stream. */
+int nfd_kv_hash(nfd_ctx *ctx, int stream, unsigned long long *h);
+
+/* Copy one frame's K and V of one layer to dev fp32 buffers [n_heads, T, head_dim]
+ * (either may be NULL).  `frame` is absolute; it must be a cached frame still in
+ * the ring or one of the scratch frames of the last pass. */
+int nfd_kv_read(nfd_ctx *ctx, int stream, int layer, int frame, float *k_out, float *v_out);
+
+/* Block-wise causal attention alone (Section 3.1), for kernel-level tests and
+ * timing.  q dev [n_heads, n_q_frames*T, head_dim]; k, v dev
+ * [n_heads, n_kv_frames*T, head_dim] in the context's storage type (bf16 or
+ * fp32).  Query frame j is frame number (n_kv_frames - n_q_frames + j) of the
+ * key sequence and sees key frames max(0, that - window) .. that.  out: dev,
+ * storage type, [n_q_frames*T, n_heads*head_dim].  The data are first copied
+ * into cache pages of batch slot 0 (which is reset), then the same attention
+ * kernel the forward pass uses runs on them.
+ * n_kv_frames <= W + k_max, n_q_frames <= k_max. */
+int nfd_attention(nfd_ctx *ctx, const void *q, const void *k, const void *v, int n_q_frames, int n_kv_frames,
+                  int window, void *out);
+
+/* Device-side status latch: 0, or the first NFD_E_* a kernel recorded.
+ * Synchronises the stream. */
+int nfd_status(nfd_ctx *ctx);
+
+/* Number of kernels the library launched (or replayed inside graphs) since
+ * creation. */
+long long nfd_launch_count(nfd_ctx *ctx);
+
+/* Run-time switches, for tests and profiling: "graph" 0/1 (replay CUDA graphs
+ * or launch kernels directly), "fast" 0/1 (tensor-core kernels or the plain
+ * validation kernels; bf16 only).  Returns NFD_E_RANGE for unknown names. */
+int nfd_set_option(nfd_ctx *ctx, const char *name, int value);
+
+const char *nfd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NFD_H_ */

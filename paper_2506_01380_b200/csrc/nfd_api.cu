@@ -1,0 +1,705 @@
+// libnfd host side: context, weight repacking, frame-paged KV cache bookkeeping,
+// pass construction, CUDA-graph capture / replay and the C ABI of include/nfd.h.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <map>
+#include <new>
+#include <vector>
+
+#include "nfd_kernels.cuh"
+#include "nfd_fast.cuh"
+
+#define CK(call)                                                                                   \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess) {                                                                   \
+            fprintf(stderr, "libnfd: %s failed: %s (%s:%d)\n", #call, cudaGetErrorString(e_),      \
+                    __FILE__, __LINE__);                                                           \
+            return NFD_E_CUDA;                                                                     \
+        }                                                                                          \
+    } while (0)
+
+#define RET(expr)                  \
+    do {                           \
+        int r_ = (expr);           \
+        if (r_ != NFD_OK) return r_; \
+    } while (0)
+
+struct GraphEntry {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    cudaGraphNode_t param_node = nullptr;
+    long long launches = 0;
+};
+
+struct nfd_ctx {
+    nfd_cfg cfg;
+    Dims D;
+    cudaStream_t st = nullptr;
+    bool bf16_mode = false;
+    size_t esz = 4;
+    bool use_graph = true, fast = true;
+    long long launches = 0;
+    std::vector<void *> allocs;
+
+    // repacked weights: matrices [out][in], storage type
+    void *w_pe = nullptr, *b_pe = nullptr, *w_t1 = nullptr, *b_t1 = nullptr, *w_t2 = nullptr, *b_t2 = nullptr;
+    void *a_emb = nullptr, *w_fmod = nullptr, *b_fmod = nullptr, *w_out = nullptr, *b_out = nullptr;
+    std::vector<void *> w_mod, b_mod, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2;
+    // device arrays of pointers for the GEMV kernels
+    void **dp_wmod = nullptr, **dp_bmod = nullptr, **dp_t1 = nullptr, **dp_t2 = nullptr, **dp_fmod = nullptr;
+    RopeTab *d_rope = nullptr;
+
+    void *kc = nullptr, *vc = nullptr;          // [n_streams][L][R][H][T][dh]
+    float *z = nullptr;                         // residual stream [Nq_max][d]
+    void *hbuf = nullptr, *qbuf = nullptr, *abuf = nullptr, *mbuf = nullptr;
+    float *emb = nullptr, *h1 = nullptr, *sc = nullptr, *mod = nullptr, *fmod = nullptr;
+    float *xp = nullptr, *vbuf = nullptr;       // sampler state, velocity
+    StepParams *d_sp = nullptr;
+    StepParams h_sp;
+    unsigned long long *d_hash = nullptr;
+    int *d_status = nullptr;
+    FastState fs;
+
+    std::vector<int> n_committed, n_tentative;
+    std::map<int, GraphEntry> graphs;
+
+    size_t frame_elems() const { return (size_t)cfg.latent_c * cfg.latent_h * cfg.latent_w; }
+    int n_total(int s) const { return n_committed[s] + n_tentative[s]; }
+};
+
+// ---------------------------------------------------------------------------
+static int dev_alloc(nfd_ctx *c, void **p, size_t bytes) {
+    *p = nullptr;
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(p, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return NFD_E_NOMEM;
+    }
+    c->allocs.push_back(*p);
+    return NFD_OK;
+}
+
+template <typename TS>
+static int repack_matrix(nfd_ctx *c, const void *src, int n_in, int n_out, void **dst, bool transpose) {
+    if (!src) return NFD_E_NULLPTR;
+    RET(dev_alloc(c, dst, (size_t)n_in * n_out * sizeof(TS)));
+    if (transpose) {
+        dim3 grid((n_out + 31) / 32, (n_in + 31) / 32), block(32, 8);
+        k_transpose<TS><<<grid, block, 0, c->st>>>((const TS *)src, (TS *)*dst, n_in, n_out);
+        CK(cudaGetLastError());
+    } else {
+        CK(cudaMemcpyAsync(*dst, src, (size_t)n_in * n_out * sizeof(TS), cudaMemcpyDeviceToDevice, c->st));
+    }
+    return NFD_OK;
+}
+
+template <typename TS> static int repack_all(nfd_ctx *c, const nfd_weights *w) {
+    const nfd_cfg &g = c->cfg;
+    const int d = g.d_model, P = c->D.P, L = g.n_layers, dm = g.d_mlp;
+    RET(repack_matrix<TS>(c, w->w_pe, P, d, &c->w_pe, true));
+    RET(repack_matrix<TS>(c, w->b_pe, 1, d, &c->b_pe, false));
+    RET(repack_matrix<TS>(c, w->w_t1, 256, d, &c->w_t1, true));
+    RET(repack_matrix<TS>(c, w->b_t1, 1, d, &c->b_t1, false));
+    RET(repack_matrix<TS>(c, w->w_t2, d, d, &c->w_t2, true));
+    RET(repack_matrix<TS>(c, w->b_t2, 1, d, &c->b_t2, false));
+    RET(repack_matrix<TS>(c, w->a_emb, g.n_actions, d, &c->a_emb, false));
+    RET(repack_matrix<TS>(c, w->w_fmod, d, 2 * d, &c->w_fmod, true));
+    RET(repack_matrix<TS>(c, w->b_fmod, 1, 2 * d, &c->b_fmod, false));
+    RET(repack_matrix<TS>(c, w->w_out, d, P, &c->w_out, true));
+    RET(repack_matrix<TS>(c, w->b_out, 1, P, &c->b_out, false));
+    if (!w->w_mod || !w->b_mod || !w->w_qkv || !w->b_qkv || !w->w_o || !w->b_o || !w->w_fc1 || !w->b_fc1 ||
+        !w->w_fc2 || !w->b_fc2)
+        return NFD_E_NULLPTR;
+    c->w_mod.resize(L), c->b_mod.resize(L), c->w_qkv.resize(L), c->b_qkv.resize(L), c->w_o.resize(L);
+    c->b_o.resize(L), c->w_fc1.resize(L), c->b_fc1.resize(L), c->w_fc2.resize(L), c->b_fc2.resize(L);
+    for (int l = 0; l < L; ++l) {
+        RET(repack_matrix<TS>(c, w->w_mod[l], d, 6 * d, &c->w_mod[l], true));
+        RET(repack_matrix<TS>(c, w->b_mod[l], 1, 6 * d, &c->b_mod[l], false));
+        RET(repack_matrix<TS>(c, w->w_qkv[l], d, 3 * d, &c->w_qkv[l], true));
+        RET(repack_matrix<TS>(c, w->b_qkv[l], 1, 3 * d, &c->b_qkv[l], false));
+        RET(repack_matrix<TS>(c, w->w_o[l], d, d, &c->w_o[l], true));
+        RET(repack_matrix<TS>(c, w->b_o[l], 1, d, &c->b_o[l], false));
+        RET(repack_matrix<TS>(c, w->w_fc1[l], d, dm, &c->w_fc1[l], true));
+        RET(repack_matrix<TS>(c, w->b_fc1[l], 1, dm, &c->b_fc1[l], false));
+        RET(repack_matrix<TS>(c, w->w_fc2[l], dm, d, &c->w_fc2[l], true));
+        RET(repack_matrix<TS>(c, w->b_fc2[l], 1, d, &c->b_fc2[l], false));
+    }
+    return NFD_OK;
+}
+
+static int upload_ptrs(nfd_ctx *c, const std::vector<void *> &v, void ***dst) {
+    RET(dev_alloc(c, (void **)dst, v.size() * sizeof(void *)));
+    CK(cudaMemcpyAsync(*dst, v.data(), v.size() * sizeof(void *), cudaMemcpyHostToDevice, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return NFD_OK;
+}
+
+static int validate_cfg(const nfd_cfg &g) {
+    if (g.n_layers < 1 || g.d_model < 128 || g.d_model > 8192 || g.d_model % 128) return NFD_E_BADCFG;
+    if (g.n_heads < 1 || g.n_heads * g.head_dim != g.d_model) return NFD_E_BADCFG;
+    if (g.head_dim != 32 && g.head_dim != 64 && g.head_dim != 128) return NFD_E_BADCFG;
+    if (g.d_mlp < 2 || g.d_mlp % 2) return NFD_E_BADCFG;
+    if (g.latent_c < 1 || g.latent_h < 1 || g.latent_w < 1 || g.patch < 1) return NFD_E_BADCFG;
+    if (g.latent_h % g.patch || g.latent_w % g.patch) return NFD_E_BADCFG;
+    int P = g.latent_c * g.patch * g.patch;
+    if (P % 2 || P > 1024) return NFD_E_BADCFG;
+    if ((size_t)g.latent_c * g.latent_h * g.latent_w % 4) return NFD_E_BADCFG;
+    if (g.n_actions < 1 || g.ctx_frames < 0 || g.ctx_frames > 4096) return NFD_E_BADCFG;
+    if (g.max_spec < 1 || g.max_spec > 8) return NFD_E_BADCFG;
+    if (g.n_streams < 1 || g.n_streams > 1024) return NFD_E_BADCFG;
+    if (g.dtype != NFD_DTYPE_FP32 && g.dtype != NFD_DTYPE_BF16) return NFD_E_BADCFG;
+    if (g.norm != 0 && g.norm != 1) return NFD_E_BADCFG;
+    if (g.act != 0) return NFD_E_BADCFG;
+    if (g.rope_t < 0 || g.rope_h < 0 || g.rope_w < 0 || (g.rope_t | g.rope_h | g.rope_w) & 1) return NFD_E_BADCFG;
+    if (g.rope_t + g.rope_h + g.rope_w != g.head_dim) return NFD_E_BADCFG;
+    if (!(g.rope_theta > 0.f) || !(g.norm_eps > 0.f) || !(g.sigma_d > 0.f)) return NFD_E_BADCFG;
+    if (!(g.t_ctx_trig >= 0.f) || !(g.t_ctx_trig < 1.5707963f)) return NFD_E_BADCFG;
+    if (g.n_steps < 1 || g.n_steps > 64) return NFD_E_BADCFG;
+    return NFD_OK;
+}
+
+static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
+
+// ---------------------------------------------------------------------------
+// One forward pass, enqueued on the context's stream.
+// ---------------------------------------------------------------------------
+#define LAUNCH(c, kern, grid, block, smem, ...)                 \
+    do {                                                        \
+        kern<<<grid, block, smem, (c)->st>>>(__VA_ARGS__);      \
+        (c)->launches++;                                        \
+    } while (0)
+
+template <typename TS, typename Epi>
+static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind) {
+    if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, c->D.T, A, Wt, M, N, K, epi, tc_kind)) {
+        c->launches++;
+        return;
+    }
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    LAUNCH(c, (k_gemm_simple<TS, Epi>), grid, 256, 0, c->d_sp, c->D.T, A, Wt, N, K, epi);
+}
+
+template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int layer) {
+    const Dims &D = c->D;
+    if (fast_attention<TS>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, D, nf, layer, (const TS *)c->qbuf,
+                           (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf)) {
+        c->launches += fast_attention_launches();
+        return;
+    }
+    long long warps = (long long)nf * D.T * D.H;
+    int grid = (int)((warps + 3) / 4);
+    if (D.dh == 32)
+        LAUNCH(c, (k_attn_simple<TS, 32>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf, (const TS *)c->kc,
+               (const TS *)c->vc, (TS *)c->abuf);
+    else if (D.dh == 64)
+        LAUNCH(c, (k_attn_simple<TS, 64>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf, (const TS *)c->kc,
+               (const TS *)c->vc, (TS *)c->abuf);
+    else
+        LAUNCH(c, (k_attn_simple<TS, 128>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf,
+               (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
+}
+
+// Kernels after k_set_params.  nf and kind are fixed per captured graph.
+template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
+    const Dims &D = c->D;
+    const int d = D.d, L = D.L, M = nf * D.T;
+    const StepParams *sp = c->d_sp;
+    const size_t mod_row = (size_t)L * 6 * d;
+    // conditioning
+    LAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
+    LAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
+           (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, c->emb, c->h1, 256, d, (size_t)d, (size_t)0);
+    LAUNCH(c, (k_gemv<TS, GEMV_T2>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t2,
+           (const TS *const *)(c->dp_t2 + 1), (const TS *)c->a_emb, c->h1, c->sc, d, d, (size_t)d, (size_t)0);
+    LAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((6 * d + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wmod,
+           (const TS *const *)c->dp_bmod, (const TS *)nullptr, c->sc, c->mod, d, 6 * d, mod_row, (size_t)6 * d);
+    if (kind == 0)
+        LAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((2 * d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_fmod,
+               (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, c->sc, c->fmod, d, 2 * d, (size_t)2 * d,
+               (size_t)0);
+    // tokens
+    LAUNCH(c, (k_patch_embed<TS>), M, 256, D.P * sizeof(float), sp, D, (const TS *)c->w_pe, (const TS *)c->b_pe,
+           c->z);
+    const int ln_grid = (M + 7) / 8;
+    for (int l = 0; l < L; ++l) {
+        const float *modl = c->mod + (size_t)l * 6 * d;
+        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0, (size_t)d);
+        EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l};
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV);
+        if (kind == 1 && l == L - 1) break;      // a commit only needs the K/V of every layer
+        launch_attention<TS>(c, nf, l);
+        EpiGateRes<TS> eo{sp, (const TS *)c->b_o[l], c->z, modl + 2 * d, mod_row, D};
+        launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES);
+        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)3 * d,
+               (size_t)4 * d);
+        EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm};
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU);
+        EpiGateRes<TS> e2{sp, (const TS *)c->b_fc2[l], c->z, modl + 5 * d, mod_row, D};
+        launch_gemm<TS>(c, (const TS *)c->mbuf, (const TS *)c->w_fc2[l], M, d, D.dm, e2, TC_RES);
+    }
+    if (kind == 0) {
+        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, c->fmod, (size_t)2 * d, (size_t)0,
+               (size_t)d);
+        EpiFinal<TS> ef{sp, (const TS *)c->b_out, D};
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_out, M, D.P, d, ef, TC_NONE);
+    }
+}
+
+static void enqueue_body_any(nfd_ctx *c, int nf, int kind) {
+    if (c->bf16_mode)
+        enqueue_body<bf16>(c, nf, kind);
+    else
+        enqueue_body<float>(c, nf, kind);
+}
+
+// Run the pass described by c->h_sp.
+static int run_pass(nfd_ctx *c) {
+    const int nf = c->h_sp.nf, kind = c->h_sp.kind;
+    if (!c->use_graph || c->st == nullptr) {
+        LAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        enqueue_body_any(c, nf, kind);
+        CK(cudaGetLastError());
+        return NFD_OK;
+    }
+    const int key = kind * 64 + nf + (c->fast ? 0 : 4096);
+    auto it = c->graphs.find(key);
+    if (it == c->graphs.end()) {
+        GraphEntry ge;
+        long long before = c->launches;
+        CK(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
+        LAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        enqueue_body_any(c, nf, kind);
+        cudaError_t e = cudaStreamEndCapture(c->st, &ge.graph);
+        ge.launches = c->launches - before;
+        c->launches = before;
+        if (e != cudaSuccess || !ge.graph) {
+            fprintf(stderr, "libnfd: graph capture failed: %s\n", cudaGetErrorString(e));
+            cudaGetLastError();
+            return NFD_E_CUDA;
+        }
+        size_t n_roots = 0;
+        CK(cudaGraphGetRootNodes(ge.graph, nullptr, &n_roots));
+        if (n_roots != 1) {
+            fprintf(stderr, "libnfd: captured graph has %zu root nodes, expected 1\n", n_roots);
+            cudaGraphDestroy(ge.graph);
+            return NFD_E_CUDA;
+        }
+        CK(cudaGraphGetRootNodes(ge.graph, &ge.param_node, &n_roots));
+        CK(cudaGraphInstantiate(&ge.exec, ge.graph, 0));
+        it = c->graphs.emplace(key, ge).first;
+    }
+    GraphEntry &ge = it->second;
+    void *args[2] = {(void *)&c->h_sp, (void *)&c->d_sp};
+    cudaKernelNodeParams kp;
+    memset(&kp, 0, sizeof(kp));
+    kp.func = (void *)k_set_params;
+    kp.gridDim = dim3(1, 1, 1);
+    kp.blockDim = dim3(256, 1, 1);
+    kp.sharedMemBytes = 0;
+    kp.kernelParams = args;
+    kp.extra = nullptr;
+    CK(cudaGraphExecKernelNodeSetParams(ge.exec, ge.param_node, &kp));
+    CK(cudaGraphLaunch(ge.exec, c->st));
+    c->launches += ge.launches;
+    return NFD_OK;
+}
+
+// Fill c->h_sp for a pass over n streams x k frames.
+//   actions: per stream (per_frame_actions = false) or per frame.
+static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, const float *t, const int *actions,
+                      bool per_frame_actions, int kind, const float *x_a, float alpha, const float *x_b, float beta,
+                      float *v_out) {
+    const nfd_cfg &g = c->cfg;
+    if (n < 1 || k < 1 || offset < 0 || offset + k > g.max_spec) return NFD_E_RANGE;
+    if ((long long)n * k > NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;
+    for (int i = 0; i < n; ++i) {
+        if (streams[i] < 0 || streams[i] >= g.n_streams) return NFD_E_RANGE;
+        for (int j = 0; j < i; ++j)
+            if (streams[j] == streams[i]) return NFD_E_RANGE;
+    }
+    StepParams &p = c->h_sp;
+    memset(&p, 0, sizeof(p));
+    p.nf = n * k;
+    p.kind = kind;
+    p.x_a = x_a, p.x_b = x_b, p.alpha = alpha, p.beta = beta, p.v_out = v_out;
+    int nc = 0;
+    for (int i = 0; i < n; ++i) {
+        for (int j = 0; j < k; ++j) {
+            int a = per_frame_actions ? actions[i * k + j] : actions[i];
+            if (a < 0 || a >= g.n_actions) return NFD_E_RANGE;
+            if (!(t[i] >= 0.f) || !(t[i] <= 1.f)) return NFD_E_RANGE;
+            int row = -1;
+            for (int r = 0; r < nc; ++r)
+                if (p.cd[r].action == a && p.cd[r].t == t[i]) row = r;
+            if (row < 0) {
+                row = nc++;
+                p.cd[row].t = t[i];
+                p.cd[row].action = a;
+            }
+            FrameDesc &f = p.fr[i * k + j];
+            f.stream = streams[i];
+            f.frame = c->n_total(streams[i]) + offset + j;
+            f.win_first = f.frame - g.ctx_frames > 0 ? f.frame - g.ctx_frames : 0;
+            f.cond_row = row;
+        }
+    }
+    p.nc = nc;
+    return NFD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------
+extern "C" {
+
+const char *nfd_strerror(int code) {
+    switch (code) {
+        case NFD_OK: return "ok";
+        case NFD_E_BADCFG: return "bad configuration";
+        case NFD_E_NULLPTR: return "null pointer";
+        case NFD_E_ALIGN: return "pointer not 16-byte aligned";
+        case NFD_E_RANGE: return "argument out of range";
+        case NFD_E_STATE: return "call not allowed in this cache state";
+        case NFD_E_NOMEM: return "out of memory";
+        case NFD_E_CUDA: return "CUDA error";
+        case NFD_E_TIMEOUT: return "device-side wait timed out";
+        case NFD_E_DEVICE: return "device-side check failed";
+        default: return "unknown error";
+    }
+}
+
+int nfd_destroy(nfd_ctx *c) {
+    if (!c) return NFD_E_NULLPTR;
+    cudaStreamSynchronize(c->st);
+    for (auto &kv : c->graphs) {
+        if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+        if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
+    }
+    fast_destroy(c->fs);
+    for (void *p : c->allocs) cudaFree(p);
+    delete c;
+    return NFD_OK;
+}
+
+int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cuda_stream) {
+    if (!out || !w || !cfg) return NFD_E_NULLPTR;
+    *out = nullptr;
+    RET(validate_cfg(*cfg));
+    nfd_ctx *c = new (std::nothrow) nfd_ctx();
+    if (!c) return NFD_E_NOMEM;
+    c->cfg = *cfg;
+    c->st = (cudaStream_t)cuda_stream;
+    c->bf16_mode = cfg->dtype == NFD_DTYPE_BF16;
+    c->esz = c->bf16_mode ? 2 : 4;
+    Dims &D = c->D;
+    D.L = cfg->n_layers, D.d = cfg->d_model, D.H = cfg->n_heads, D.dh = cfg->head_dim, D.dm = cfg->d_mlp;
+    D.C = cfg->latent_c, D.Hl = cfg->latent_h, D.Wl = cfg->latent_w, D.p = cfg->patch;
+    D.th = D.Hl / D.p, D.tw = D.Wl / D.p, D.T = D.th * D.tw, D.P = D.C * D.p * D.p;
+    D.R = cfg->ctx_frames + cfg->max_spec, D.W = cfg->ctx_frames, D.n_streams = cfg->n_streams;
+    D.norm = cfg->norm, D.eps = cfg->norm_eps, D.t_scale = cfg->t_scale;
+    D.page_elems = (size_t)D.H * D.T * D.dh;
+    c->n_committed.assign(cfg->n_streams, 0);
+    c->n_tentative.assign(cfg->n_streams, 0);
+    if (getenv("NFD_NO_GRAPH")) c->use_graph = false;
+    if (getenv("NFD_NO_FAST")) c->fast = false;
+
+    int rc = c->bf16_mode ? repack_all<bf16>(c, w) : repack_all<float>(c, w);
+    const int NF = NFD_MAX_PASS_FRAMES;
+    const size_t Mmax = (size_t)NF * D.T;
+    auto A = [&](void **p, size_t bytes) { if (rc == NFD_OK) rc = dev_alloc(c, p, bytes); };
+    const size_t cache_elems = (size_t)D.n_streams * D.L * D.R * D.page_elems;
+    A(&c->kc, cache_elems * c->esz);
+    A(&c->vc, cache_elems * c->esz);
+    A((void **)&c->z, Mmax * D.d * 4);
+    A(&c->hbuf, Mmax * D.d * c->esz);
+    A(&c->qbuf, Mmax * D.d * c->esz);
+    A(&c->abuf, Mmax * D.d * c->esz);
+    A(&c->mbuf, Mmax * D.dm * c->esz);
+    A((void **)&c->emb, (size_t)NF * 256 * 4);
+    A((void **)&c->h1, (size_t)NF * D.d * 4);
+    A((void **)&c->sc, (size_t)NF * D.d * 4);
+    A((void **)&c->mod, (size_t)NF * D.L * 6 * D.d * 4);
+    A((void **)&c->fmod, (size_t)NF * 2 * D.d * 4);
+    A((void **)&c->xp, (size_t)NF * c->frame_elems() * 4);
+    A((void **)&c->vbuf, (size_t)NF * c->frame_elems() * 4);
+    A((void **)&c->d_sp, sizeof(StepParams));
+    A((void **)&c->d_hash, 8);
+    A((void **)&c->d_status, 4);
+    A((void **)&c->d_rope, sizeof(RopeTab));
+    if (rc == NFD_OK) {
+        std::vector<void *> v;
+        v = c->w_mod; rc = upload_ptrs(c, v, &c->dp_wmod);
+        if (rc == NFD_OK) { v = c->b_mod; rc = upload_ptrs(c, v, &c->dp_bmod); }
+        if (rc == NFD_OK) { v = {c->w_t1, c->b_t1}; rc = upload_ptrs(c, v, &c->dp_t1); }
+        if (rc == NFD_OK) { v = {c->w_t2, c->b_t2}; rc = upload_ptrs(c, v, &c->dp_t2); }
+        if (rc == NFD_OK) { v = {c->w_fmod, c->b_fmod}; rc = upload_ptrs(c, v, &c->dp_fmod); }
+    }
+    if (rc == NFD_OK) {
+        RopeTab rt;
+        memset(&rt, 0, sizeof(rt));
+        int pi = 0;
+        const int dims[3] = {cfg->rope_t, cfg->rope_h, cfg->rope_w};
+        for (int ax = 0; ax < 3; ++ax)
+            for (int i = 0; i < dims[ax] / 2; ++i, ++pi) {
+                rt.axis[pi] = ax;
+                rt.freq[pi] = (float)pow((double)cfg->rope_theta, -2.0 * i / (double)dims[ax]);
+            }
+        cudaError_t e = cudaMemcpyAsync(c->d_rope, &rt, sizeof(rt), cudaMemcpyHostToDevice, c->st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->kc, 0, cache_elems * c->esz, c->st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->vc, 0, cache_elems * c->esz, c->st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4, c->st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->st);
+        if (e != cudaSuccess) {
+            fprintf(stderr, "libnfd: create: %s\n", cudaGetErrorString(e));
+            rc = NFD_E_CUDA;
+        }
+    }
+    if (rc == NFD_OK) rc = fast_create(c->fs, D, c->bf16_mode, c->st, c->d_status);
+    if (rc != NFD_OK) {
+        nfd_destroy(c);
+        return rc;
+    }
+    *out = c;
+    return NFD_OK;
+}
+
+int nfd_reset(nfd_ctx *c, int stream) {
+    if (!c) return NFD_E_NULLPTR;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    c->n_committed[stream] = 0;
+    c->n_tentative[stream] = 0;
+    return NFD_OK;
+}
+
+static int check_io(const void *a, const void *b) {
+    if (!a || !b) return NFD_E_NULLPTR;
+    if (!aligned16(a) || !aligned16(b)) return NFD_E_ALIGN;
+    return NFD_OK;
+}
+
+int nfd_denoise_step_batched(nfd_ctx *c, int n, const int *streams, const float *x_t, int k, const float *t,
+                             const int *actions, float *v_out) {
+    if (!c || !streams || !t || !actions) return NFD_E_NULLPTR;
+    RET(check_io(x_t, v_out));
+    RET(build_pass(c, n, streams, k, 0, t, actions, false, 0, x_t, 1.0f, nullptr, 0.f, v_out));
+    return run_pass(c);
+}
+
+int nfd_denoise_step_at(nfd_ctx *c, int stream, int offset, const float *x_t, int k, float t, int action,
+                        float *v_out) {
+    if (!c) return NFD_E_NULLPTR;
+    RET(check_io(x_t, v_out));
+    RET(build_pass(c, 1, &stream, k, offset, &t, &action, false, 0, x_t, 1.0f, nullptr, 0.f, v_out));
+    return run_pass(c);
+}
+
+int nfd_denoise_step(nfd_ctx *c, int stream, const float *x_t, int k, float t, int action, float *v_out) {
+    return nfd_denoise_step_at(c, stream, 0, x_t, k, t, action, v_out);
+}
+
+// Commit pass over n streams x k frames; actions per frame.
+static int commit_pass(nfd_ctx *c, int n, const int *streams, int k, const int *actions, const float *x0,
+                       const float *ctx_noise, bool tentative) {
+    const double tc = c->cfg.t_ctx_trig, sd = c->cfg.sigma_d;
+    const double sn = sin(tc), cs = cos(tc);
+    const double t_fm = sn / (sn + cs);
+    const double scale = sqrt(t_fm * t_fm + (1 - t_fm) * (1 - t_fm));
+    std::vector<float> t(n, (float)t_fm);
+    RET(build_pass(c, n, streams, k, 0, t.data(), actions, true, 1, x0, (float)(cs * scale / sd), ctx_noise,
+                   (float)(sn * scale), nullptr));
+    RET(run_pass(c));
+    for (int i = 0; i < n; ++i) (tentative ? c->n_tentative : c->n_committed)[streams[i]] += k;
+    return NFD_OK;
+}
+
+int nfd_commit_frame(nfd_ctx *c, int stream, const float *x0, int n, const int *actions, const float *ctx_noise) {
+    if (!c || !x0 || !actions) return NFD_E_NULLPTR;
+    if (!aligned16(x0) || !aligned16(ctx_noise)) return NFD_E_ALIGN;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    if (c->n_tentative[stream] != 0) return NFD_E_STATE;
+    return commit_pass(c, 1, &stream, n, actions, x0, ctx_noise, false);
+}
+
+int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const int *actions, const float *noise,
+                          const float *ctx_noise, float *x0_out) {
+    if (!c || !streams || !actions) return NFD_E_NULLPTR;
+    RET(check_io(noise, x0_out));
+    if (!aligned16(ctx_noise)) return NFD_E_ALIGN;
+    if (n < 1 || k < 1 || k > c->cfg.max_spec || (long long)n * k > NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;
+    for (int i = 0; i < n; ++i) {
+        if (streams[i] < 0 || streams[i] >= c->cfg.n_streams) return NFD_E_RANGE;
+        if (actions[i] < 0 || actions[i] >= c->cfg.n_actions) return NFD_E_RANGE;
+        if (c->n_tentative[streams[i]] != 0) return NFD_E_STATE;
+    }
+    const int S = c->cfg.n_steps;
+    const double sd = c->cfg.sigma_d;
+    const size_t ne = (size_t)n * k * c->frame_elems();
+    const int eg = (int)((ne + 255) / 256);
+    // Section 4.1 "Sampling": start from pure noise at t' = pi/2
+    LAUNCH(c, k_axpby, eg, 256, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
+    std::vector<float> tv(n);
+    for (int s = 0; s < S; ++s) {
+        const double tp = 0.5 * M_PI * (double)(S - s) / (double)S;
+        const double sn = sin(tp), cs = cos(tp);
+        const double t = sn / (sn + cs);
+        const double alpha = sqrt(t * t + (1 - t) * (1 - t)) / sd;
+        for (int i = 0; i < n; ++i) tv[i] = (float)t;
+        RET(build_pass(c, n, streams, k, 0, tv.data(), actions, false, 0, c->xp, (float)alpha, nullptr, 0.f,
+                       c->vbuf));
+        RET(run_pass(c));
+        // clean estimate sigma_d (x_in - t v), then re-noise to the next timestep
+        const float *z = nullptr;
+        double cn = 0, sn_next = 0;
+        if (s + 1 < S) {
+            const double tpn = 0.5 * M_PI * (double)(S - s - 1) / (double)S;
+            z = noise + (size_t)(s + 1) * ne;
+            cn = cos(tpn), sn_next = sin(tpn) * sd;
+        }
+        LAUNCH(c, k_sampler_post, eg, 256, 0, c->xp, c->vbuf, z, x0_out, (float)(sd * alpha), (float)(-sd * t),
+               (float)cn, (float)sn_next, ne);
+    }
+    CK(cudaGetLastError());
+    std::vector<int> fa((size_t)n * k);
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < k; ++j) fa[i * k + j] = actions[i];
+    return commit_pass(c, n, streams, k, fa.data(), x0_out, ctx_noise, true);
+}
+
+int nfd_speculate(nfd_ctx *c, int stream, int k, int action, const float *noise, const float *ctx_noise,
+                  float *x0_out) {
+    return nfd_speculate_batched(c, 1, &stream, k, &action, noise, ctx_noise, x0_out);
+}
+
+int nfd_rollback(nfd_ctx *c, int stream, int n_accept) {
+    if (!c) return NFD_E_NULLPTR;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    if (n_accept < 0 || n_accept > c->n_tentative[stream]) return NFD_E_RANGE;
+    c->n_committed[stream] += n_accept;
+    c->n_tentative[stream] = 0;
+    return NFD_OK;
+}
+
+int nfd_kv_state(nfd_ctx *c, int stream, int *n_committed, int *n_tentative, int *window_first) {
+    if (!c) return NFD_E_NULLPTR;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    if (n_committed) *n_committed = c->n_committed[stream];
+    if (n_tentative) *n_tentative = c->n_tentative[stream];
+    int wf = c->n_total(stream) - c->cfg.ctx_frames;
+    if (window_first) *window_first = wf > 0 ? wf : 0;
+    return NFD_OK;
+}
+
+int nfd_kv_hash(nfd_ctx *c, int stream, unsigned long long *h) {
+    if (!c || !h) return NFD_E_NULLPTR;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    const int total = c->n_total(stream);
+    const int first = total - c->cfg.ctx_frames > 0 ? total - c->cfg.ctx_frames : 0;
+    const int count = total - first;
+    CK(cudaMemsetAsync(c->d_hash, 0, 8, c->st));
+    if (count > 0) {
+        if (c->bf16_mode)
+            LAUNCH(c, (k_kv_hash<bf16>), 592, 256, 0, c->D, (const bf16 *)c->kc, (const bf16 *)c->vc, stream, first,
+                   count, c->d_hash);
+        else
+            LAUNCH(c, (k_kv_hash<float>), 592, 256, 0, c->D, (const float *)c->kc, (const float *)c->vc, stream,
+                   first, count, c->d_hash);
+        CK(cudaGetLastError());
+    }
+    unsigned long long v = 0;
+    CK(cudaMemcpyAsync(&v, c->d_hash, 8, cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    v ^= 0x9e3779b97f4a7c15ULL * (unsigned long long)(c->n_committed[stream] + 1);
+    v ^= 0xc2b2ae3d27d4eb4fULL * (unsigned long long)(c->n_tentative[stream] + 1);
+    *h = v;
+    return NFD_OK;
+}
+
+int nfd_kv_read(nfd_ctx *c, int stream, int layer, int frame, float *k_out, float *v_out) {
+    if (!c) return NFD_E_NULLPTR;
+    if (stream < 0 || stream >= c->cfg.n_streams || layer < 0 || layer >= c->cfg.n_layers) return NFD_E_RANGE;
+    const int total = c->n_total(stream);
+    if (frame < 0 || frame >= total + c->cfg.max_spec || frame < total + c->cfg.max_spec - c->D.R) return NFD_E_RANGE;
+    const int grid = (int)((c->D.page_elems + 255) / 256);
+    for (int which = 0; which < 2; ++which) {
+        float *o = which ? v_out : k_out;
+        const void *cache = which ? c->vc : c->kc;
+        if (!o) continue;
+        if (c->bf16_mode)
+            LAUNCH(c, (k_kv_read<bf16>), grid, 256, 0, c->D, (const bf16 *)cache, stream, layer, frame, o);
+        else
+            LAUNCH(c, (k_kv_read<float>), grid, 256, 0, c->D, (const float *)cache, stream, layer, frame, o);
+    }
+    CK(cudaGetLastError());
+    return NFD_OK;
+}
+
+int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n_q, int n_kv, int window,
+                  void *out) {
+    if (!c || !q || !out) return NFD_E_NULLPTR;
+    if ((k == nullptr) != (v == nullptr)) return NFD_E_NULLPTR;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return NFD_E_ALIGN;
+    if (n_q < 1 || n_q > c->cfg.max_spec || n_kv < n_q || n_kv > c->D.R || window < 0) return NFD_E_RANGE;
+    const Dims &D = c->D;
+    c->n_committed[0] = 0;
+    c->n_tentative[0] = 0;
+    const size_t fill = (size_t)n_kv * D.page_elems;
+    if (k) {
+        const int grid = (int)((fill + 255) / 256);
+        if (c->bf16_mode) {
+            LAUNCH(c, (k_kv_fill<bf16>), grid, 256, 0, D, (bf16 *)c->kc, 0, (const bf16 *)k, n_kv);
+            LAUNCH(c, (k_kv_fill<bf16>), grid, 256, 0, D, (bf16 *)c->vc, 0, (const bf16 *)v, n_kv);
+        } else {
+            LAUNCH(c, (k_kv_fill<float>), grid, 256, 0, D, (float *)c->kc, 0, (const float *)k, n_kv);
+            LAUNCH(c, (k_kv_fill<float>), grid, 256, 0, D, (float *)c->vc, 0, (const float *)v, n_kv);
+        }
+    }
+    const size_t qbytes = (size_t)n_q * D.T * D.d * c->esz;
+    CK(cudaMemcpyAsync(c->qbuf, q, qbytes, cudaMemcpyDeviceToDevice, c->st));
+    StepParams &p = c->h_sp;
+    memset(&p, 0, sizeof(p));
+    p.nf = n_q;
+    p.nc = 1;
+    for (int j = 0; j < n_q; ++j) {
+        p.fr[j].stream = 0;
+        p.fr[j].frame = n_kv - n_q + j;
+        p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
+    }
+    LAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp);
+    if (c->bf16_mode)
+        launch_attention<bf16>(c, n_q, 0);
+    else
+        launch_attention<float>(c, n_q, 0);
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(out, c->abuf, qbytes, cudaMemcpyDeviceToDevice, c->st));
+    return NFD_OK;
+}
+
+int nfd_status(nfd_ctx *c) {
+    if (!c) return NFD_E_NULLPTR;
+    int s = 0;
+    CK(cudaMemcpyAsync(&s, c->d_status, 4, cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return s;
+}
+
+long long nfd_launch_count(nfd_ctx *c) { return c ? c->launches : 0; }
+
+int nfd_set_option(nfd_ctx *c, const char *name, int value) {
+    if (!c || !name) return NFD_E_NULLPTR;
+    if (!strcmp(name, "graph")) {
+        c->use_graph = value != 0;
+        return NFD_OK;
+    }
+    if (!strcmp(name, "fast")) {
+        c->fast = value != 0;
+        return NFD_OK;
+    }
+    return NFD_E_RANGE;
+}
+
+}  // extern "C"

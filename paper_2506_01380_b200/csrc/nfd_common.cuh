@@ -1,0 +1,81 @@
+// Shared device-side types and helpers of libnfd (CUDA, sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "nfd.h"
+
+typedef __nv_bfloat16 bf16;
+
+// One frame of a forward pass.
+struct FrameDesc {
+    int stream;      // batch slot
+    int frame;       // absolute frame index (RoPE position, ring slot = frame % R)
+    int win_first;   // first frame this one attends to (>= 0, >= frame - W)
+    int cond_row;    // row of the conditioning / modulation tables
+};
+
+// One distinct (FM time, action) pair of a pass.
+struct CondDesc {
+    float t;
+    int action;
+};
+
+// Everything that changes from pass to pass.  Written to device memory by the
+// first kernel of every pass so that a captured graph can be replayed with new
+// values (cache position, timestep, action, I/O pointers).
+struct StepParams {
+    int nf;                 // frames in this pass (tokens = nf * T)
+    int nc;                 // distinct conditioning rows
+    int kind;               // 0 denoise (all layers + velocity head), 1 commit (K/V only)
+    int layer_for_attn;     // nfd_attention: which layer's pages hold the data
+    const float *x_a;       // model input = alpha * x_a + beta * x_b
+    const float *x_b;       // may be NULL
+    float *v_out;           // [nf,C,H,W]
+    float alpha, beta;
+    FrameDesc fr[NFD_MAX_PASS_FRAMES];
+    CondDesc cd[NFD_MAX_PASS_FRAMES];
+};
+
+// Static model dimensions, passed by value to kernels.
+struct Dims {
+    int L, d, H, dh, dm;
+    int C, Hl, Wl, p, th, tw, T, P;
+    int R, W, n_streams;
+    int norm;
+    float eps, t_scale;
+    size_t page_elems;      // H*T*dh
+};
+
+#define NFD_MAX_HALF_DH 64
+// RoPE table: for pair i of the head dimension, the axis it rotates with
+// (0 frame, 1 row, 2 col) and its frequency.
+struct RopeTab {
+    float freq[NFD_MAX_HALF_DH];
+    int axis[NFD_MAX_HALF_DH];
+};
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ size_t kv_page_offset(const Dims &D, int stream, int layer, int frame) {
+    return ((size_t)(stream * D.L + layer) * D.R + (size_t)(frame % D.R)) * D.page_elems;
+}
+
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}

@@ -1,0 +1,418 @@
+// Plain CUDA kernels of libnfd: conditioning, patch embedding, adaLN norm,
+// epilogue functors shared by every GEMM, a straightforward tiled GEMM and a
+// straightforward attention kernel (both used in fp32 validation mode and as
+// the "fast = 0" path in bf16 mode), sampler glue, cache digest / read-out.
+#pragma once
+#include "nfd_common.cuh"
+
+// ---------------------------------------------------------------------------
+// Pass parameters: first kernel of every pass.
+// ---------------------------------------------------------------------------
+__global__ void k_set_params(StepParams p, StepParams *dst) {
+    const int n_words = sizeof(StepParams) / 4;
+    const int *src = reinterpret_cast<const int *>(&p);
+    int *d = reinterpret_cast<int *>(dst);
+    for (int i = threadIdx.x; i < n_words; i += blockDim.x) d[i] = src[i];
+}
+
+// ---------------------------------------------------------------------------
+// Conditioning (adaLN-zero on timestep + action, Section 3.1 "Action
+// Conditioning"): sinusoidal embedding of t_scale * t, MLP with SiLU, plus the
+// action embedding row; then per-layer modulation W_mod * SiLU(c) + b.
+// ---------------------------------------------------------------------------
+__global__ void k_temb(const StepParams *sp, float t_scale, float *emb /*[rows][256]*/) {
+    int c = blockIdx.x;
+    if (c >= sp->nc) return;
+    int i = threadIdx.x;              // 0..127
+    if (i >= 128) return;
+    // double precision: the argument reaches ~1e3 rad
+    double f = exp(-9.210340371976184 /* ln 1e4 */ * (double)i / 128.0);
+    double a = (double)t_scale * (double)sp->cd[c].t * f;
+    double s, co;
+    sincos(a, &s, &co);
+    emb[c * 256 + i] = (float)co;
+    emb[c * 256 + 128 + i] = (float)s;
+}
+
+enum { GEMV_T1 = 0, GEMV_T2 = 1, GEMV_MOD = 2 };
+
+// y[c][o] = f( sum_i Wt[o][i] * x[c][i] + b[o] ), one warp per output o, all
+// conditioning rows c.  blockIdx.y selects the layer for GEMV_MOD.
+template <typename TS, int MODE>
+__global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *const *Wt_l, const TS *const *b_l,
+                                              const TS *a_emb, const float *x, float *y, int n_in, int n_out,
+                                              size_t y_row_stride, size_t y_layer_stride) {
+    const int layer = blockIdx.y;
+    const TS *Wt = Wt_l[layer];
+    const TS *b = b_l[layer];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int o = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (o >= n_out) return;
+    const int nc = sp->nc;
+    const TS *wrow = Wt + (size_t)o * n_in;
+    for (int c = 0; c < nc; ++c) {
+        const float *xc = x + (size_t)c * n_in;
+        float acc = 0.f;
+        for (int i = lane; i < n_in; i += 32) acc = fmaf(to_f(wrow[i]), xc[i], acc);
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            float v = acc + to_f(b[o]);
+            if (MODE == GEMV_T1) v = silu_f(v);
+            if (MODE == GEMV_T2) v = silu_f(v + to_f(a_emb[(size_t)sp->cd[c].action * n_out + o]));
+            y[(size_t)c * y_row_stride + (size_t)layer * y_layer_stride + o] = v;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Patchify + embed: z[tok][o] = sum_p (alpha*x_a + beta*x_b)[patch p of tok] * Wt_pe[o][p] + b[o]
+// ---------------------------------------------------------------------------
+template <typename TS>
+__global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *Wt_pe, const TS *b_pe,
+                                                     float *z) {
+    extern __shared__ float s_patch[];
+    const int m = blockIdx.x;
+    if (m >= sp->nf * D.T) return;
+    const int j = m / D.T, tok = m % D.T;
+    const int r = tok / D.tw, c = tok % D.tw;
+    const float *xa = sp->x_a, *xb = sp->x_b;
+    const float alpha = sp->alpha, beta = sp->beta;
+    for (int p = threadIdx.x; p < D.P; p += blockDim.x) {
+        int ch = p / (D.p * D.p), py = (p / D.p) % D.p, px = p % D.p;
+        size_t idx = (((size_t)j * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
+        float v = alpha * xa[idx];
+        if (xb) v = fmaf(beta, xb[idx], v);
+        s_patch[p] = v;
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < D.d; o += blockDim.x) {
+        const TS *w = Wt_pe + (size_t)o * D.P;
+        float acc = 0.f;
+        for (int p = 0; p < D.P; ++p) acc = fmaf(s_patch[p], to_f(w[p]), acc);
+        z[(size_t)m * D.d + o] = acc + to_f(b_pe[o]);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// adaLN: out = norm(z) * (1 + scale_f) + shift_f, one warp per token.
+// ---------------------------------------------------------------------------
+template <typename TS>
+__global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, const float *z, TS *out,
+                                               const float *mod, size_t row_stride, size_t off_shift,
+                                               size_t off_scale) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (m >= sp->nf * D.T) return;
+    const int row = sp->fr[m / D.T].cond_row;
+    const float *zr = z + (size_t)m * D.d;
+    const float *sh = mod + (size_t)row * row_stride + off_shift;
+    const float *sc = mod + (size_t)row * row_stride + off_scale;
+    float s = 0.f;
+    for (int i = lane * 4; i < D.d; i += 128) {
+        float4 v = *reinterpret_cast<const float4 *>(zr + i);
+        s += (v.x + v.y) + (v.z + v.w);
+    }
+    const float inv_d = 1.0f / (float)D.d;
+    float mean = (D.norm == 0) ? warp_sum(s) * inv_d : 0.f;
+    float q = 0.f;
+    for (int i = lane * 4; i < D.d; i += 128) {
+        float4 v = *reinterpret_cast<const float4 *>(zr + i);
+        float a = v.x - mean, b = v.y - mean, c = v.z - mean, e = v.w - mean;
+        q += (a * a + b * b) + (c * c + e * e);
+    }
+    const float rstd = rsqrtf(warp_sum(q) * inv_d + D.eps);
+    for (int i = lane * 4; i < D.d; i += 128) {
+        float4 v = *reinterpret_cast<const float4 *>(zr + i);
+        float4 a = *reinterpret_cast<const float4 *>(sh + i);
+        float4 b = *reinterpret_cast<const float4 *>(sc + i);
+        TS *o = out + (size_t)m * D.d + i;
+        o[0] = from_f<TS>(fmaf((v.x - mean) * rstd, 1.0f + b.x, a.x));
+        o[1] = from_f<TS>(fmaf((v.y - mean) * rstd, 1.0f + b.y, a.y));
+        o[2] = from_f<TS>(fmaf((v.z - mean) * rstd, 1.0f + b.z, a.z));
+        o[3] = from_f<TS>(fmaf((v.w - mean) * rstd, 1.0f + b.w, a.w));
+    }
+}
+
+// ---------------------------------------------------------------------------
+// GEMM epilogues.  Each is called with one output row m and two adjacent
+// columns (n, n+1), n even, holding the fp32 accumulators.
+// ---------------------------------------------------------------------------
+// QKV: + bias, 3D RoPE on q and k (Section 3.1 "3D Positional Embedding":
+// adjacent pairs, per-axis frequencies), q -> [H][Nq][dh], k/v -> cache pages.
+template <typename TS> struct EpiQKV {
+    const StepParams *sp;
+    const TS *bias;
+    TS *q, *kc, *vc;
+    const RopeTab *rt;
+    Dims D;
+    int layer;
+    __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
+        a0 += to_f(bias[n]);
+        a1 += to_f(bias[n + 1]);
+        const int which = n / D.d, col = n % D.d;
+        const int head = col / D.dh, e = col % D.dh;
+        const int j = m / D.T, tok = m % D.T;
+        const FrameDesc fr = sp->fr[j];
+        if (which < 2) {
+            const int pi = e >> 1;
+            const int ax = rt->axis[pi];
+            const float pos = (float)(ax == 0 ? fr.frame : (ax == 1 ? tok / D.tw : tok % D.tw));
+            float sn, cs;
+            sincosf(pos * rt->freq[pi], &sn, &cs);
+            const float r0 = a0 * cs - a1 * sn, r1 = a0 * sn + a1 * cs;
+            a0 = r0;
+            a1 = r1;
+        }
+        TS *dst;
+        if (which == 0) {
+            dst = q + ((size_t)head * (sp->nf * D.T) + m) * D.dh + e;
+        } else {
+            TS *base = (which == 1) ? kc : vc;
+            dst = base + kv_page_offset(D, fr.stream, layer, fr.frame) + ((size_t)head * D.T + tok) * D.dh + e;
+        }
+        dst[0] = from_f<TS>(a0);
+        dst[1] = from_f<TS>(a1);
+    }
+};
+
+// z += gate_f * (acc + bias): residual update of the fp32 stream.
+template <typename TS> struct EpiGateRes {
+    const StepParams *sp;
+    const TS *bias;
+    float *z;
+    const float *gate;      // mod + layer offset + chunk offset
+    size_t row_stride;
+    Dims D;
+    __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
+        const int row = sp->fr[m / D.T].cond_row;
+        const float *g = gate + (size_t)row * row_stride + n;
+        float *zp = z + (size_t)m * D.d + n;
+        zp[0] = fmaf(g[0], a0 + to_f(bias[n]), zp[0]);
+        zp[1] = fmaf(g[1], a1 + to_f(bias[n + 1]), zp[1]);
+    }
+};
+
+// out = GELU(acc + bias), exact erf form.
+template <typename TS> struct EpiGelu {
+    const TS *bias;
+    TS *out;
+    int N;
+    __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
+        TS *o = out + (size_t)m * N + n;
+        o[0] = from_f<TS>(gelu_erf_f(a0 + to_f(bias[n])));
+        o[1] = from_f<TS>(gelu_erf_f(a1 + to_f(bias[n + 1])));
+    }
+};
+
+// Velocity head: + bias, unpatchify into v_out [nf,C,H,W].
+template <typename TS> struct EpiFinal {
+    const StepParams *sp;
+    const TS *bias;
+    Dims D;
+    __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
+        const int j = m / D.T, tok = m % D.T;
+        const int r = tok / D.tw, c = tok % D.tw;
+        float av[2] = {a0 + to_f(bias[n]), a1 + to_f(bias[n + 1])};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            int p = n + u;
+            int ch = p / (D.p * D.p), py = (p / D.p) % D.p, px = p % D.p;
+            size_t idx = (((size_t)j * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
+            sp->v_out[idx] = av[u];
+        }
+    }
+};
+
+// ---------------------------------------------------------------------------
+// Straightforward GEMM: C[m][n] = sum_k A[m][k] * Wt[n][k], fp32 accumulation,
+// 64x64 tile, 16-deep k slices.  M = sp->nf * T (read on the device).
+// ---------------------------------------------------------------------------
+template <typename TS, typename Epi>
+__global__ void __launch_bounds__(256) k_gemm_simple(const StepParams *sp, int T, const TS *__restrict__ A,
+                                                     const TS *__restrict__ Wt, int N, int K, Epi epi) {
+    __shared__ float As[16][64];
+    __shared__ float Bs[16][64];
+    const int M = sp->nf * T;
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    if (m0 >= M) return;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int lr = tid >> 2, lk = (tid & 3) * 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += 16) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int k = k0 + lk + u;
+            int m = m0 + lr, n = n0 + lr;
+            As[lk + u][lr] = (m < M && k < K) ? to_f(A[(size_t)m * K + k]) : 0.f;
+            Bs[lk + u][lr] = (n < N && k < K) ? to_f(Wt[(size_t)n * K + k]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float4 a = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
+            float4 b = *reinterpret_cast<const float4 *>(&Bs[kk][tx * 4]);
+            float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; j += 2) {
+            int n = n0 + tx * 4 + j;
+            if (n + 1 < N) epi(m, n, acc[i][j], acc[i][j + 1]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Straightforward block-wise causal attention (Section 3.1): one warp per
+// (query token, head); keys are walked frame page by frame page over the
+// query frame's window, so the mask is a page range and never a matrix.
+// Lanes split the head dimension; online softmax in fp32.
+// ---------------------------------------------------------------------------
+template <typename TS, int DH>
+__global__ void __launch_bounds__(128) k_attn_simple(const StepParams *sp, Dims D, int layer, const TS *q,
+                                                     const TS *kc, const TS *vc, TS *out) {
+    constexpr int R = DH / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int Nq = sp->nf * D.T;
+    const long long w = (long long)blockIdx.x * (blockDim.x >> 5) + warp;
+    if (w >= (long long)Nq * D.H) return;
+    const int m = (int)(w / D.H), h = (int)(w % D.H);
+    const FrameDesc fr = sp->fr[m / D.T];
+    float qv[R], acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        qv[r] = to_f(q[((size_t)h * Nq + m) * DH + lane + 32 * r]);
+        acc[r] = 0.f;
+    }
+    const float scale = rsqrtf((float)DH);
+    float mx = -INFINITY, l = 0.f;
+    for (int g = fr.win_first; g <= fr.frame; ++g) {
+        const size_t off = kv_page_offset(D, fr.stream, layer, g) + (size_t)h * D.T * DH;
+        const TS *kp = kc + off, *vp = vc + off;
+        for (int j = 0; j < D.T; ++j) {
+            float s = 0.f;
+#pragma unroll
+            for (int r = 0; r < R; ++r) s = fmaf(qv[r], to_f(kp[(size_t)j * DH + lane + 32 * r]), s);
+            s = warp_sum(s) * scale;
+            const float mn = fmaxf(mx, s);
+            const float corr = expf(mx - mn), p = expf(s - mn);
+            l = l * corr + p;
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[r] = fmaf(p, to_f(vp[(size_t)j * DH + lane + 32 * r]), acc[r] * corr);
+            mx = mn;
+        }
+    }
+    const float inv = 1.0f / l;
+#pragma unroll
+    for (int r = 0; r < R; ++r) out[(size_t)m * D.d + h * DH + lane + 32 * r] = from_f<TS>(acc[r] * inv);
+}
+
+// ---------------------------------------------------------------------------
+// Sampler glue (Section 4.1): elementwise.
+// ---------------------------------------------------------------------------
+// out = a*x + b*y (y may be NULL)
+__global__ void k_axpby(float *out, float a, const float *x, float b, const float *y, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float v = a * x[i];
+    if (y) v = fmaf(b, y[i], v);
+    out[i] = v;
+}
+
+// x0 = a*x' + b*v  (= sigma_d (x_in - t v));  if z: x' <- c*x0 + s*z  (re-noise to the next timestep)
+__global__ void k_sampler_post(float *xp, const float *v, const float *z, float *x0, float a, float b, float c,
+                               float s, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float e = fmaf(b, v[i], a * xp[i]);
+    x0[i] = e;
+    if (z) xp[i] = fmaf(s, z[i], c * e);
+}
+
+// ---------------------------------------------------------------------------
+// Cache read-out, fill and digest.
+// ---------------------------------------------------------------------------
+template <typename TS>
+__global__ void k_kv_read(Dims D, const TS *cache, int stream, int layer, int frame, float *out) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= D.page_elems) return;
+    out[i] = to_f(cache[kv_page_offset(D, stream, layer, frame) + i]);
+}
+
+// copy [H][n_frames*T][dh] (storage type) into pages of (stream 0, layer) frames 0..n_frames-1
+template <typename TS>
+__global__ void k_kv_fill(Dims D, TS *cache, int layer, const TS *src, int n_frames) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t total = (size_t)n_frames * D.page_elems;
+    if (i >= total) return;
+    int e = (int)(i % D.dh);
+    size_t r = i / D.dh;
+    int tok_all = (int)(r % ((size_t)n_frames * D.T));
+    int h = (int)(r / ((size_t)n_frames * D.T));
+    int f = tok_all / D.T, tok = tok_all % D.T;
+    cache[kv_page_offset(D, 0, layer, f) + ((size_t)h * D.T + tok) * D.dh + e] = src[i];
+}
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
+    x ^= x >> 33;
+    x *= 0xff51afd7ed558ccdULL;
+    x ^= x >> 33;
+    x *= 0xc4ceb9fe1a85ec53ULL;
+    x ^= x >> 33;
+    return x;
+}
+
+// Order-independent digest: sum over elements of mix(logical position, raw bits).
+// The logical position is (layer, absolute frame, K or V, offset in page), so
+// the digest does not depend on which ring slot holds a frame.
+template <typename TS>
+__global__ void k_kv_hash(Dims D, const TS *kc, const TS *vc, int stream, int first, int count,
+                          unsigned long long *acc) {
+    const size_t per_layer = (size_t)count * D.page_elems;
+    const size_t total = per_layer * D.L;
+    unsigned long long local = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        int layer = (int)(i / per_layer);
+        size_t r = i % per_layer;
+        int f = first + (int)(r / D.page_elems);
+        size_t e = r % D.page_elems;
+        size_t off = kv_page_offset(D, stream, layer, f) + e;
+        unsigned long long kb, vb;
+        if (sizeof(TS) == 2) {
+            kb = *reinterpret_cast<const unsigned short *>(kc + off);
+            vb = *reinterpret_cast<const unsigned short *>(vc + off);
+        } else {
+            kb = *reinterpret_cast<const unsigned int *>(kc + off);
+            vb = *reinterpret_cast<const unsigned int *>(vc + off);
+        }
+        unsigned long long pos = (((unsigned long long)layer * 0x100000ULL + (unsigned long long)f) << 32) ^ e;
+        local += mix64(pos * 2 + 0 + (kb << 40) + 0x9e3779b97f4a7c15ULL) + mix64((pos * 2 + 1) ^ (vb << 36));
+    }
+    atomicAdd(acc, local);
+}
+
+// transpose [rows][cols] -> [cols][rows]
+template <typename TS>
+__global__ void k_transpose(const TS *in, TS *out, int rows, int cols) {
+    __shared__ TS tile[32][33];
+    int c = blockIdx.x * 32 + threadIdx.x, r0 = blockIdx.y * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (r0 + i < rows && c < cols) tile[i][threadIdx.x] = in[(size_t)(r0 + i) * cols + c];
+    __syncthreads();
+    int r = r0 + threadIdx.x, c0 = blockIdx.x * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (c0 + i < cols && r < rows) out[(size_t)(c0 + i) * rows + r] = tile[threadIdx.x][i];
+}
