@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the NFD hot path (libnfd) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A "step" generates ONE frame of the 310M-class configuration at batch 1 with a
+16-frame KV context: 4 denoising passes (sampler glue included) plus the commit
+pass that appends the frame's K/V, i.e. one nfd_speculate(k=1) + nfd_rollback.
+Metric: frames/sec.  One JSON line is printed by rank 0.
+
+N > 1 runs N independent replicas (one stream per GPU, no collective on the
+data path): the path does not shard inside a stream.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "frames/sec at batch 1 (310M-class, 4 steps, k=1)"
+UNIT = "frames/s"
+WORKLOAD = "nfd310m: 24L d1024 16x64 heads MLP4096 GELU, 336 tokens/frame, 16-frame KV context, 4 steps + commit, k=1"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sust=d["bf16_tflops_sustained"], src="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, src="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, torch_device):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_device).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(torch_device.index or 0)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:               # no NVML: report that, never fail the bench
+            self.nv = None
+            self.err = repr(e)
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def start(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self._thr:
+            self._stop.set()
+            self._thr.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# ---------------------------------------------------------------------------
+# algorithmic work of one launch of each kernel class (k = 1 pass, steady state)
+# ---------------------------------------------------------------------------
+def class_work(cfg, T, n_ctx):
+    d, dm, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
+    M, Nk = T, (n_ctx + 1) * T
+
+    def gemm(N, K, res=False):
+        return dict(flops=2.0 * M * N * K, bytes=2.0 * (N * K + M * K + M * N) + (8.0 * M * N if res else 0.0))
+    return {
+        "gemm_qkv_rope_kvstore": gemm(3 * d, d),
+        "gemm_out_gate_res": gemm(d, d, True),
+        "gemm_fc1_gelu": gemm(dm, d),
+        "gemm_fc2_gate_res": gemm(d, dm, True),
+        "attention": dict(flops=4.0 * M * Nk * d, bytes=2.0 * (2 * Nk * d + 2 * M * d)),
+        "adaln_norm": dict(flops=8.0 * M * d, bytes=M * d * 6.0),
+        "conditioning": dict(flops=2.0 * 6 * d * d, bytes=2.0 * 6 * d * d),   # per layer-launch average
+    }
+
+
+def roofline_of(cfg, T, n_ctx, prof, pk):
+    work = class_work(cfg, T, n_ctx)
+    total = sum(ms for _, ms in prof.values()) or 1.0
+    shares = {k: round(ms / total, 4) for k, (n, ms) in prof.items() if n}
+    cand = [(ms, k) for k, (n, ms) in prof.items() if n and k in work]
+    if not cand:
+        return None, shares
+    ms, name = max(cand)
+    n = prof[name][0]
+    dur = ms / n * 1e-3
+    w = work[name]
+    t_flop, t_byte = w["flops"] / (pk["tf_sust"] * 1e12), w["bytes"] / (pk["hbm"] * 1e9)
+    if name == "conditioning":
+        # one class covers several small GEMV launches; report the modulation GEMV bytes of a pass
+        w = dict(flops=0.0, bytes=2.0 * 6 * cfg["d_model"] ** 2 * cfg["n_layers"])
+        dur = ms / (n / 5.0) * 1e-3
+        t_flop, t_byte = 0.0, 1.0
+    if t_flop >= t_byte:
+        ach, peak, unit, bound = w["flops"] / dur / 1e12, pk["tf_sust"], "TFLOP/s", "tensor"
+    else:
+        ach, peak, unit, bound = w["bytes"] / dur / 1e9, pk["hbm"], "GB/s", "hbm"
+    return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
+            "frac": round(ach / peak, 4), "peak_source": pk["src"] + (" (sustained)" if bound == "tensor" else ""),
+            "avg_launch_us": round(dur * 1e6, 2), "share_of_step": shares.get(name), "traffic": None}, shares
+
+
+# ---------------------------------------------------------------------------
+def oracle_sample(cfg, n_passes_denoise=1, seed=0):
+    """Time the fp64 oracle, as it stands, on one forward pass (k=1) over a full
+    16-frame context whose K/V pages are filled with N(0,1) values (building the
+    context with the oracle itself would take minutes and is not what is timed)."""
+    import numpy as np
+    from oracle import nfd_oracle as O
+    from paper_2506_01380_b200 import inputs as I
+    w = I.make_weights(cfg, seed)
+    orc = O.NFDOracle(cfg, w)
+    rng = np.random.default_rng(1)
+    W, H, T, dh = cfg["ctx_frames"], cfg["n_heads"], I.tokens_per_frame(cfg), cfg["head_dim"]
+    for l in range(cfg["n_layers"]):
+        for f in range(W):
+            orc.kv[l][f] = (rng.standard_normal((H, T, dh)), rng.standard_normal((H, T, dh)))
+    orc.n_committed = W
+    x = I.make_latents(cfg, 1, 2).astype(np.float64)
+    times = []
+    for _ in range(n_passes_denoise):
+        t0 = time.perf_counter()
+        orc.denoise_step(x, 0.7, 1)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count()
+
+
+def run_reference(args):
+    """Reference arm = the oracle on the host cores (the paper ships no code)."""
+    from paper_2506_01380_b200 import inputs as I
+    import numpy  # noqa: F401  (loads BLAS so that the thread count is known)
+    cfg = I.make_cfg("nfd310m")
+    steps = max(1, min(args.steps, 6))
+    warm = max(0, min(args.warmup, 1))
+    times = oracle_sample(cfg, warm + steps)[warm:]
+    t_pass = sum(times) / len(times)
+    passes_per_frame = cfg["n_steps"] + 1
+    value = 1.0 / (passes_per_frame * t_pass)
+    sample = (f"each step = 1 forward pass (k=1, 16-frame context of random K/V pages); a frame = "
+              f"{passes_per_frame} passes, value extrapolated as 1/({passes_per_frame}*t_pass); "
+              f"steps capped at {steps}")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warm, "ms_per_step": t_pass * passes_per_frame * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def torch_weights(cfg, device, seed):
+    """Seeded N(0, 0.02^2) weights generated on the device (bf16-rounded by the upload)."""
+    import torch
+    from paper_2506_01380_b200 import inputs as I
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return {n: torch.randn(s, generator=g, device=device, dtype=torch.float32) * 0.02
+            for n, s in I.weight_shapes(cfg).items()}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-extras", action="store_true", help="skip the k=4, e2e, profile and CPU legs")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return 0
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2506_01380_b200 import inputs as I
+    from paper_2506_01380_b200.nfd import NFD
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    cfg = I.make_cfg("nfd310m")
+    S, W, T = cfg["n_steps"], cfg["ctx_frames"], I.tokens_per_frame(cfg)
+    fs = I.frame_shape(cfg)
+    nfd = NFD(cfg, torch_weights(cfg, device, seed=0), device=str(device))
+    K, Wm = args.steps, args.warmup
+    gen = torch.Generator(device=device)
+    gen.manual_seed(1000 + rank)
+
+    def randn(*shape):
+        return torch.randn(*shape, generator=gen, device=device, dtype=torch.float32)
+
+    def fill_prompt():
+        nfd.reset(0)
+        acts = I.make_actions_uniform(cfg, W, 7 + rank)
+        for i in range(0, W, 4):
+            nfd.commit_frame(randn(4, *fs), acts[i:i + 4], randn(4, *fs))
+
+    def barrier():
+        torch.cuda.synchronize(device)
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize(device)
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---------------- device-resident leg (the headline `value`) ----------------
+    fill_prompt()
+    n_all = K + Wm
+    noise = randn(n_all, S, 1, *fs)
+    cnoise = randn(n_all, 1, *fs)
+    actions = I.make_actions_uniform(cfg, n_all, rank)
+    x0 = torch.empty((1,) + fs, device=device)
+    with torch.cuda.stream(nfd.stream):
+        for i in range(Wm):
+            nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
+            nfd.rollback(1)
+        barrier()
+        clocks = ClockSampler(device)
+        clocks.start()
+        l0 = nfd.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(nfd.stream)
+        for i in range(Wm, n_all):
+            nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
+            nfd.rollback(1)
+        e1.record(nfd.stream)
+        barrier()
+        clk = clocks.stop()
+        ms = max_over_ranks(e0.elapsed_time(e1))
+        launches = nfd.launch_count() - l0
+    assert nfd.status() == 0
+    value = world * K / (ms * 1e-3)
+    pk = peaks()
+    line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": "inputs larger than L2: 604 MB of weights + 528 MB of KV pages are streamed every pass",
+                       "passes_per_step": S + 1, "cuda_graph": True},
+            "clocks": clk, "gpu_launches": int(launches)}
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        # ---------------- end-to-end leg: host buffers in, host frame out ----------------
+        n_e = min(K, 32)
+        h_noise = torch.randn(n_e, S, 1, *fs).pin_memory()
+        h_cn = torch.randn(n_e, 1, *fs).pin_memory()
+        h_out = torch.empty((1,) + fs).pin_memory()
+        d_noise, d_cn = torch.empty((S, 1) + fs, device=device), torch.empty((1,) + fs, device=device)
+        with torch.cuda.stream(nfd.stream):
+            torch.cuda.synchronize(device)
+            e0.record(nfd.stream)
+            for i in range(n_e):
+                d_noise.copy_(h_noise[i], non_blocking=True)
+                d_cn.copy_(h_cn[i], non_blocking=True)
+                nfd.speculate(1, actions[i], d_noise, d_cn, out=x0)
+                nfd.rollback(1)
+                h_out.copy_(x0, non_blocking=True)
+                nfd.stream.synchronize()          # the caller needs the frame before choosing the next action
+            e1.record(nfd.stream)
+            torch.cuda.synchronize(device)
+        ms_e = e0.elapsed_time(e1)
+        line["e2e"] = {"value": round(n_e / (ms_e * 1e-3), 3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(d_noise.numel() * 4 + d_cn.numel() * 4),
+                       "d2h_bytes_per_step": int(x0.numel() * 4), "steps": n_e}
+
+        # ---------------- speculative k = 4 on a Markov action chain ----------------
+        from paper_2506_01380_b200.nfd import accepted_frames
+        k = 4
+        n_frames = max(K, 64)
+        chain = I.make_action_chain(cfg, n_frames + k + 8, seed=0, p_repeat=0.8)
+        fill_prompt()
+        noise4, cn4 = randn(S, k, *fs), randn(k, *fs)
+        x04 = torch.empty((k,) + fs, device=device)
+        with torch.cuda.stream(nfd.stream):
+            for _ in range(3):
+                nfd.speculate(k, chain[0], noise4, cn4, out=x04)
+                nfd.rollback(1)
+            fill_prompt()
+            torch.cuda.synchronize(device)
+            i = spec = acc = passes = 0
+            e0.record(nfd.stream)
+            while i < n_frames:
+                nfd.speculate(k, chain[i], noise4, cn4, out=x04)
+                n_acc = accepted_frames(chain, i, k)
+                nfd.rollback(n_acc)
+                spec += k
+                acc += n_acc
+                passes += 1
+                i += n_acc
+            e1.record(nfd.stream)
+            torch.cuda.synchronize(device)
+        ms4 = e0.elapsed_time(e1)
+        line["spec_k4"] = {"accepted_frames_per_s": round(acc / (ms4 * 1e-3), 3), "acceptance_rate": round(acc / spec, 4),
+                           "accepted_per_pass": round(acc / passes, 4), "ms_per_speculate": round(ms4 / passes, 4),
+                           "p_repeat": 0.8, "frames": acc}
+
+        # ---------------- per-kernel timing (events around every launch) ----------------
+        fill_prompt()
+        with torch.cuda.stream(nfd.stream):
+            nfd.profile_begin()
+            for i in range(4):
+                nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
+                nfd.rollback(1)
+            prof = nfd.profile_end()
+        roof, shares = roofline_of(cfg, T, W, prof, pk)
+        line["roofline"] = roof
+        line["kernel_time_shares"] = shares
+        # whole-pass roofline: the slower of FLOPs at the bf16 peak and bytes at HBM bandwidth
+        d, dm, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
+        gemm_params = L * (4 * d * d + 2 * d * dm)
+        flops = 2.0 * T * gemm_params + 4.0 * T * (W + 1) * T * d * L
+        byts = 2.0 * gemm_params + 2.0 * 2 * L * W * T * d
+        t_roof = max(flops / (pk["tf_sust"] * 1e12), byts / (pk["hbm"] * 1e9))
+        line["pass_roofline"] = {"flops_per_pass": flops, "bytes_per_pass": byts,
+                                 "roofline_frames_per_s": round(1.0 / ((S + 1) * t_roof), 1),
+                                 "frac": round(value / (1.0 / ((S + 1) * t_roof)), 4), "peak_source": pk["src"]}
+
+        # ---------------- the oracle on this machine's host cores ----------------
+        t_or = oracle_sample(cfg, 2)
+        t_pass = min(t_or)
+        line["cpu_baseline"] = {"value": round(1.0 / ((S + 1) * t_pass), 5), "unit": UNIT, "cores": cpu_threads(),
+                                "kind": "oracle",
+                                "sample": f"1 forward pass (k=1, 16-frame context of random K/V pages) = "
+                                          f"{t_pass:.2f} s; frames/s extrapolated as 1/({S + 1} passes)"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

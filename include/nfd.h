@@ -178,6 +178,18 @@ int nfd_status(nfd_ctx *ctx);
  * creation. */
 long long nfd_launch_count(nfd_ctx *ctx);
 
+/* Per-kernel timing.  Between nfd_profile_begin and nfd_profile_end every
+ * kernel is launched directly (no graph replay) with a CUDA event before and
+ * after it on the context's stream.  nfd_profile_end synchronises and returns,
+ * per kernel class id < n_classes, the number of launches and their summed
+ * device time in milliseconds (host arrays of n_classes entries).  Class ids
+ * run 0 .. nfd_profile_class_count()-1 and are named by
+ * nfd_profile_class_name. */
+int nfd_profile_begin(nfd_ctx *ctx);
+int nfd_profile_end(nfd_ctx *ctx, int n_classes, long long *n_launches, float *total_ms);
+int nfd_profile_class_count(void);
+const char *nfd_profile_class_name(int id);
+
 /* Run-time switches, for tests and profiling: "graph" 0/1 (replay CUDA graphs
  * or launch kernels directly), "fast" 0/1 (tensor-core kernels or the plain
  * validation kernels; bf16 only).  Returns NFD_E_RANGE for unknown names. */

@@ -67,6 +67,13 @@ struct nfd_ctx {
     std::vector<int> n_committed, n_tentative;
     std::map<int, GraphEntry> graphs;
 
+    // per-kernel-class timing (nfd_profile_begin / nfd_profile_end)
+    bool prof = false;
+    int cls = 0;
+    std::vector<cudaEvent_t> prof_ev;       // pairs: start, stop
+    std::vector<int> prof_cls;
+    size_t prof_used = 0;
+
     size_t frame_elems() const { return (size_t)cfg.latent_c * cfg.latent_h * cfg.latent_w; }
     int n_total(int s) const { return n_committed[s] + n_tentative[s]; }
 };
@@ -168,15 +175,45 @@ static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
 // ---------------------------------------------------------------------------
 // One forward pass, enqueued on the context's stream.
 // ---------------------------------------------------------------------------
+enum { CLS_PARAMS = 0, CLS_COND, CLS_PATCH, CLS_ADALN, CLS_GEMM_QKV, CLS_ATTN, CLS_GEMM_O, CLS_GEMM_FC1,
+       CLS_GEMM_FC2, CLS_HEAD, CLS_SAMPLER, CLS_CACHE, CLS_COUNT };
+static const char *const kClassNames[CLS_COUNT] = {"params", "conditioning", "patch_embed", "adaln_norm",
+                                                   "gemm_qkv_rope_kvstore", "attention", "gemm_out_gate_res",
+                                                   "gemm_fc1_gelu", "gemm_fc2_gate_res", "velocity_head",
+                                                   "sampler", "cache_util"};
+
+static void prof_mark(nfd_ctx *c, bool stop) {
+    if (!c->prof) return;
+    if (!stop) {
+        if (c->prof_used + 2 > c->prof_ev.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                cudaEventCreate(&e);
+                c->prof_ev.push_back(e);
+            }
+        }
+        c->prof_cls.resize(c->prof_ev.size() / 2);
+        c->prof_cls[c->prof_used / 2] = c->cls;
+        cudaEventRecord(c->prof_ev[c->prof_used], c->st);
+    } else {
+        cudaEventRecord(c->prof_ev[c->prof_used + 1], c->st);
+        c->prof_used += 2;
+    }
+}
+
 #define LAUNCH(c, kern, grid, block, smem, ...)                 \
     do {                                                        \
+        prof_mark((c), false);                                  \
         kern<<<grid, block, smem, (c)->st>>>(__VA_ARGS__);      \
+        prof_mark((c), true);                                   \
         (c)->launches++;                                        \
     } while (0)
 
 template <typename TS, typename Epi>
 static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind) {
+    prof_mark(c, false);
     if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, c->D.T, A, Wt, M, N, K, epi, tc_kind)) {
+        prof_mark(c, true);
         c->launches++;
         return;
     }
@@ -186,8 +223,11 @@ static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int
 
 template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int layer) {
     const Dims &D = c->D;
+    c->cls = CLS_ATTN;
+    prof_mark(c, false);
     if (fast_attention<TS>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, D, nf, layer, (const TS *)c->qbuf,
                            (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf)) {
+        prof_mark(c, true);
         c->launches += fast_attention_launches();
         return;
     }
@@ -211,6 +251,7 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
     // conditioning
+    c->cls = CLS_COND;
     LAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
     LAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
            (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, c->emb, c->h1, 256, d, (size_t)d, (size_t)0);
@@ -223,26 +264,34 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
                (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, c->sc, c->fmod, d, 2 * d, (size_t)2 * d,
                (size_t)0);
     // tokens
+    c->cls = CLS_PATCH;
     LAUNCH(c, (k_patch_embed<TS>), M, 256, D.P * sizeof(float), sp, D, (const TS *)c->w_pe, (const TS *)c->b_pe,
            c->z);
     const int ln_grid = (M + 7) / 8;
     for (int l = 0; l < L; ++l) {
         const float *modl = c->mod + (size_t)l * 6 * d;
+        c->cls = CLS_ADALN;
         LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0, (size_t)d);
         EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l};
+        c->cls = CLS_GEMM_QKV;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV);
         if (kind == 1 && l == L - 1) break;      // a commit only needs the K/V of every layer
         launch_attention<TS>(c, nf, l);
         EpiGateRes<TS> eo{sp, (const TS *)c->b_o[l], c->z, modl + 2 * d, mod_row, D};
+        c->cls = CLS_GEMM_O;
         launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES);
+        c->cls = CLS_ADALN;
         LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)3 * d,
                (size_t)4 * d);
         EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm};
+        c->cls = CLS_GEMM_FC1;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU);
         EpiGateRes<TS> e2{sp, (const TS *)c->b_fc2[l], c->z, modl + 5 * d, mod_row, D};
+        c->cls = CLS_GEMM_FC2;
         launch_gemm<TS>(c, (const TS *)c->mbuf, (const TS *)c->w_fc2[l], M, d, D.dm, e2, TC_RES);
     }
     if (kind == 0) {
+        c->cls = CLS_HEAD;
         LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, c->fmod, (size_t)2 * d, (size_t)0,
                (size_t)d);
         EpiFinal<TS> ef{sp, (const TS *)c->b_out, D};
@@ -260,7 +309,8 @@ static void enqueue_body_any(nfd_ctx *c, int nf, int kind) {
 // Run the pass described by c->h_sp.
 static int run_pass(nfd_ctx *c) {
     const int nf = c->h_sp.nf, kind = c->h_sp.kind;
-    if (!c->use_graph || c->st == nullptr) {
+    if (!c->use_graph || c->st == nullptr || c->prof) {
+        c->cls = CLS_PARAMS;
         LAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
         enqueue_body_any(c, nf, kind);
         CK(cudaGetLastError());
@@ -381,6 +431,7 @@ int nfd_destroy(nfd_ctx *c) {
         if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
     }
     fast_destroy(c->fs);
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     for (void *p : c->allocs) cudaFree(p);
     delete c;
     return NFD_OK;
@@ -541,6 +592,7 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
     const size_t ne = (size_t)n * k * c->frame_elems();
     const int eg = (int)((ne + 255) / 256);
     // Section 4.1 "Sampling": start from pure noise at t' = pi/2
+    c->cls = CLS_SAMPLER;
     LAUNCH(c, k_axpby, eg, 256, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
     std::vector<float> tv(n);
     for (int s = 0; s < S; ++s) {
@@ -560,6 +612,7 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
             z = noise + (size_t)(s + 1) * ne;
             cn = cos(tpn), sn_next = sin(tpn) * sd;
         }
+        c->cls = CLS_SAMPLER;
         LAUNCH(c, k_sampler_post, eg, 256, 0, c->xp, c->vbuf, z, x0_out, (float)(sd * alpha), (float)(-sd * t),
                (float)cn, (float)sn_next, ne);
     }
@@ -601,6 +654,7 @@ int nfd_kv_hash(nfd_ctx *c, int stream, unsigned long long *h) {
     const int first = total - c->cfg.ctx_frames > 0 ? total - c->cfg.ctx_frames : 0;
     const int count = total - first;
     CK(cudaMemsetAsync(c->d_hash, 0, 8, c->st));
+    c->cls = CLS_CACHE;
     if (count > 0) {
         if (c->bf16_mode)
             LAUNCH(c, (k_kv_hash<bf16>), 592, 256, 0, c->D, (const bf16 *)c->kc, (const bf16 *)c->vc, stream, first,
@@ -625,6 +679,7 @@ int nfd_kv_read(nfd_ctx *c, int stream, int layer, int frame, float *k_out, floa
     const int total = c->n_total(stream);
     if (frame < 0 || frame >= total + c->cfg.max_spec || frame < total + c->cfg.max_spec - c->D.R) return NFD_E_RANGE;
     const int grid = (int)((c->D.page_elems + 255) / 256);
+    c->cls = CLS_CACHE;
     for (int which = 0; which < 2; ++which) {
         float *o = which ? v_out : k_out;
         const void *cache = which ? c->vc : c->kc;
@@ -648,6 +703,7 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
     c->n_committed[0] = 0;
     c->n_tentative[0] = 0;
     const size_t fill = (size_t)n_kv * D.page_elems;
+    c->cls = CLS_CACHE;
     if (k) {
         const int grid = (int)((fill + 255) / 256);
         if (c->bf16_mode) {
@@ -669,6 +725,7 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
         p.fr[j].frame = n_kv - n_q + j;
         p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
     }
+    c->cls = CLS_PARAMS;
     LAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp);
     if (c->bf16_mode)
         launch_attention<bf16>(c, n_q, 0);
@@ -688,6 +745,34 @@ int nfd_status(nfd_ctx *c) {
 }
 
 long long nfd_launch_count(nfd_ctx *c) { return c ? c->launches : 0; }
+
+int nfd_profile_begin(nfd_ctx *c) {
+    if (!c) return NFD_E_NULLPTR;
+    CK(cudaStreamSynchronize(c->st));
+    c->prof = true;
+    c->prof_used = 0;
+    return NFD_OK;
+}
+
+int nfd_profile_end(nfd_ctx *c, int n_classes, long long *n_launches, float *total_ms) {
+    if (!c || !n_launches || !total_ms) return NFD_E_NULLPTR;
+    if (!c->prof) return NFD_E_STATE;
+    c->prof = false;
+    CK(cudaStreamSynchronize(c->st));
+    for (int i = 0; i < n_classes; ++i) n_launches[i] = 0, total_ms[i] = 0.f;
+    for (size_t i = 0; i + 1 < c->prof_used; i += 2) {
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]));
+        int k = c->prof_cls[i / 2];
+        if (k >= 0 && k < n_classes) n_launches[k]++, total_ms[k] += ms;
+    }
+    c->prof_used = 0;
+    return NFD_OK;
+}
+
+int nfd_profile_class_count(void) { return CLS_COUNT; }
+
+const char *nfd_profile_class_name(int id) { return (id >= 0 && id < CLS_COUNT) ? kClassNames[id] : ""; }
 
 int nfd_set_option(nfd_ctx *c, const char *name, int value) {
     if (!c || !name) return NFD_E_NULLPTR;

@@ -83,10 +83,12 @@ def frame_shape(cfg):
 def round_bf16(a: np.ndarray) -> np.ndarray:
     """Round an fp32 array to the nearest bf16 value (ties to even), kept as fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)
-    u = a.view(np.uint32).astype(np.uint64)
-    lsb = (u >> 16) & 1
-    u = (u + 0x7FFF + lsb) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+    u = a.view(np.uint32).copy()
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    lsb += np.uint32(0x7FFF)
+    u += lsb                      # finite inputs cannot overflow 32 bits here
+    u &= np.uint32(0xFFFF0000)
+    return u.view(np.float32).reshape(a.shape)
 
 
 def weight_shapes(cfg) -> dict:

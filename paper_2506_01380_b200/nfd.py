@@ -42,7 +42,8 @@ class NfdWeights(C.Structure):
 EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_denoise_step_at",
            "nfd_denoise_step_batched", "nfd_commit_frame", "nfd_speculate", "nfd_speculate_batched",
            "nfd_rollback", "nfd_kv_state", "nfd_kv_hash", "nfd_kv_read", "nfd_attention", "nfd_status",
-           "nfd_launch_count", "nfd_set_option", "nfd_strerror"]
+           "nfd_launch_count", "nfd_set_option", "nfd_strerror", "nfd_profile_begin", "nfd_profile_end",
+           "nfd_profile_class_count", "nfd_profile_class_name"]
 
 
 class NfdError(RuntimeError):
@@ -81,6 +82,11 @@ def load():
     lib.nfd_launch_count.argtypes = [vp]
     lib.nfd_launch_count.restype = C.c_longlong
     lib.nfd_set_option.argtypes = [vp, C.c_char_p, C.c_int]
+    lib.nfd_profile_begin.argtypes = [vp]
+    lib.nfd_profile_end.argtypes = [vp, C.c_int, C.POINTER(C.c_longlong), fp]
+    lib.nfd_profile_class_count.argtypes = []
+    lib.nfd_profile_class_name.argtypes = [C.c_int]
+    lib.nfd_profile_class_name.restype = C.c_char_p
     lib.nfd_strerror.argtypes = [C.c_int]
     lib.nfd_strerror.restype = C.c_char_p
     _lib = lib
@@ -108,6 +114,19 @@ def _floats(v):
 def _check(code: int, what: str):
     if code != 0:
         raise NfdError(code, what)
+
+
+def accepted_frames(true_actions, i: int, k: int) -> int:
+    """Host-side verification of a speculation (Section 4.2): frames i .. i+k-1
+    were generated under true_actions[i].  Returns how many leading frames were
+    generated under their true action (always >= 1); pass it to rollback()."""
+    first = true_actions[i]
+    n = 1
+    for j in range(i + 1, min(i + k, len(true_actions))):
+        if true_actions[j] != first:
+            break
+        n += 1
+    return n
 
 
 class NFD:
@@ -262,6 +281,16 @@ class NFD:
 
     def launch_count(self) -> int:
         return self.lib.nfd_launch_count(self._h)
+
+    def profile_begin(self):
+        _check(self.lib.nfd_profile_begin(self._h), "nfd_profile_begin")
+
+    def profile_end(self) -> dict:
+        """{class name: (launches, total milliseconds)}"""
+        n = self.lib.nfd_profile_class_count()
+        cnt, ms = (C.c_longlong * n)(), (C.c_float * n)()
+        _check(self.lib.nfd_profile_end(self._h, n, cnt, ms), "nfd_profile_end")
+        return {self.lib.nfd_profile_class_name(i).decode(): (int(cnt[i]), float(ms[i])) for i in range(n)}
 
     def set_option(self, name: str, value: int):
         _check(self.lib.nfd_set_option(self._h, name.encode(), int(value)), "nfd_set_option")

@@ -54,3 +54,13 @@ def test_strerror_needs_no_gpu():
     lib = N.load()
     assert lib.nfd_strerror(0) == b"ok"
     assert lib.nfd_strerror(-5) == b"call not allowed in this cache state"
+
+
+def test_host_side_acceptance_rule_matches_oracle():
+    import itertools
+    from oracle.nfd_oracle import accepted_count
+    for n in range(1, 7):
+        for acts in itertools.product([0, 1, 2], repeat=n):
+            for k in range(1, 5):
+                for i in range(n):
+                    assert N.accepted_frames(list(acts), i, k) == accepted_count(list(acts), i, k)
