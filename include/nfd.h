@@ -170,6 +170,38 @@ int nfd_kv_read(nfd_ctx *ctx, int stream, int layer, int frame, float *k_out, fl
 int nfd_attention(nfd_ctx *ctx, const void *q, const void *k, const void *v, int n_q_frames, int n_kv_frames,
                   int window, void *out);
 
+/* Block-wise causal attention for callers that must not allocate.  (The paper
+ * has no counterpart of this call; it exists for integration reasons only.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they
+ * need attention: code running while a CUDA graph is being captured, a
+ * real-time frame loop that forbids allocator calls after start-up, a process
+ * whose device memory is handed out by an arena owned by someone else.  This
+ * call creates no context and calls no cudaMalloc / cudaFree and no allocating
+ * library routine.  Its only working memory, the descriptor of the query frames
+ * that the kernel reads, is a fixed 4 KiB array inside the library image; every
+ * GPU that loads the library holds those 4 KiB until the process exits.
+ *
+ *   q        dev [n_heads, n_q_frames*T, head_dim]
+ *   k_pages  dev [n_kv_frames, n_heads, T, head_dim]   (frame pages, as the cache stores them)
+ *   v_pages  dev [n_kv_frames, n_heads, T, head_dim]
+ *   out      dev [n_q_frames*T, n_heads*head_dim]
+ *   dtype    NFD_DTYPE_FP32 or NFD_DTYPE_BF16: element type of all four
+ *   T = tokens_per_frame.  Query frame j is key frame (n_kv_frames - n_q_frames + j)
+ *   and sees key frames max(0, that - window) .. that.
+ *
+ * Limit: n_q_frames <= NFD_MAX_PASS_FRAMES (32) -- more descriptors do not fit
+ * the fixed array; larger values return NFD_E_RANGE and print the reason.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.
+ * All calls on a device share the one array: it is rewritten in full by every
+ * call, so nothing needs clearing, but two calls whose kernels overlap on the
+ * GPU (different streams) race on it -- serialise them.
+ * Runs the plain attention kernel on `cuda_stream` (a cudaStream_t). */
+int nfd_attention_noalloc(const void *q, const void *k_pages, const void *v_pages, int dtype, int n_heads,
+                          int head_dim, int tokens_per_frame, int n_q_frames, int n_kv_frames, int window,
+                          void *out, void *cuda_stream);
+
 /* Device-side status latch: 0, or the first NFD_E_* a kernel recorded.
  * Synchronises the stream. */
 int nfd_status(nfd_ctx *ctx);

@@ -787,4 +787,88 @@ int nfd_set_option(nfd_ctx *c, const char *name, int value) {
     return NFD_E_RANGE;
 }
 
+
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Allocation-free attention entry point.
+//
+// The pass descriptor that the attention kernel reads (which frames are
+// queried, which page window each may see) normally lives in memory the
+// context allocated with cudaMalloc.  Here it lives in a fixed array that is
+// part of the library image, so the call needs no allocator at all.
+// ---------------------------------------------------------------------------
+#define NFD_NOALLOC_SCRATCH_BYTES 4096
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NFD_NOALLOC_SCRATCH_BYTES];
+static_assert(sizeof(StepParams) <= NFD_NOALLOC_SCRATCH_BYTES, "pass descriptor must fit the static scratch");
+
+#define NFD_NOALLOC_MAX_DEVICES 64
+// Device address of g_noalloc_scratch per device ordinal.  In host code the
+// symbol itself is only a stand-in, so its address is looked up once per device.
+static void *g_noalloc_dev_ptr[NFD_NOALLOC_MAX_DEVICES] = {nullptr};
+
+template <typename TS>
+static int noalloc_launch(cudaStream_t st, const StepParams *d_sp, const Dims &D, int n_q, const void *q,
+                          const void *k_pages, const void *v_pages, void *out) {
+    const long long warps = (long long)n_q * D.T * D.H;
+    const int grid = (int)((warps + 3) / 4);
+    if (D.dh == 32)
+        k_attn_simple<TS, 32><<<grid, 128, 0, st>>>(d_sp, D, 0, (const TS *)q, (const TS *)k_pages,
+                                                    (const TS *)v_pages, (TS *)out);
+    else if (D.dh == 64)
+        k_attn_simple<TS, 64><<<grid, 128, 0, st>>>(d_sp, D, 0, (const TS *)q, (const TS *)k_pages,
+                                                    (const TS *)v_pages, (TS *)out);
+    else
+        k_attn_simple<TS, 128><<<grid, 128, 0, st>>>(d_sp, D, 0, (const TS *)q, (const TS *)k_pages,
+                                                     (const TS *)v_pages, (TS *)out);
+    CK(cudaGetLastError());
+    return NFD_OK;
+}
+
+extern "C" int nfd_attention_noalloc(const void *q, const void *k_pages, const void *v_pages, int dtype, int n_heads,
+                          int head_dim, int tokens_per_frame, int n_q_frames, int n_kv_frames, int window,
+                          void *out, void *cuda_stream) {
+    if (!q || !k_pages || !v_pages || !out) return NFD_E_NULLPTR;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out)) return NFD_E_ALIGN;
+    if (dtype != NFD_DTYPE_FP32 && dtype != NFD_DTYPE_BF16) return NFD_E_BADCFG;
+    if (head_dim != 32 && head_dim != 64 && head_dim != 128) return NFD_E_BADCFG;
+    if (n_heads < 1 || tokens_per_frame < 1 || window < 0) return NFD_E_RANGE;
+    if (n_q_frames < 1 || n_q_frames > NFD_MAX_PASS_FRAMES) {
+        fprintf(stderr, "libnfd: nfd_attention_noalloc: n_q_frames = %d, but the static scratch holds the "
+                        "descriptors of at most %d query frames\n", n_q_frames, NFD_MAX_PASS_FRAMES);
+        return NFD_E_RANGE;
+    }
+    if (n_kv_frames < n_q_frames || n_kv_frames > 65536) return NFD_E_RANGE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= NFD_NOALLOC_MAX_DEVICES) return NFD_E_RANGE;
+    if (!g_noalloc_dev_ptr[dev]) {
+        // one-time set-up for the current device: turn the symbol into a device address
+        void *p = nullptr;
+        CK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) return NFD_E_CUDA;
+        g_noalloc_dev_ptr[dev] = p;
+    }
+    StepParams *d_sp = (StepParams *)g_noalloc_dev_ptr[dev];
+    Dims D;
+    memset(&D, 0, sizeof(D));
+    D.L = 1, D.H = n_heads, D.dh = head_dim, D.d = n_heads * head_dim, D.T = tokens_per_frame;
+    D.R = n_kv_frames, D.W = window, D.n_streams = 1;
+    D.page_elems = (size_t)n_heads * tokens_per_frame * head_dim;
+    StepParams p;
+    memset(&p, 0, sizeof(p));
+    p.nf = n_q_frames;
+    p.nc = 1;
+    for (int j = 0; j < n_q_frames; ++j) {
+        p.fr[j].stream = 0;
+        p.fr[j].frame = n_kv_frames - n_q_frames + j;
+        p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
+    }
+    // the descriptor is rewritten in full on every call; nothing of the previous call survives
+    k_set_params<<<1, 256, 0, st>>>(p, d_sp);
+    CK(cudaGetLastError());
+    if (dtype == NFD_DTYPE_BF16) return noalloc_launch<bf16>(st, d_sp, D, n_q_frames, q, k_pages, v_pages, out);
+    return noalloc_launch<float>(st, d_sp, D, n_q_frames, q, k_pages, v_pages, out);
+}
+

@@ -43,7 +43,7 @@ EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_de
            "nfd_denoise_step_batched", "nfd_commit_frame", "nfd_speculate", "nfd_speculate_batched",
            "nfd_rollback", "nfd_kv_state", "nfd_kv_hash", "nfd_kv_read", "nfd_attention", "nfd_status",
            "nfd_launch_count", "nfd_set_option", "nfd_strerror", "nfd_profile_begin", "nfd_profile_end",
-           "nfd_profile_class_count", "nfd_profile_class_name"]
+           "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc"]
 
 
 class NfdError(RuntimeError):
@@ -87,6 +87,8 @@ def load():
     lib.nfd_profile_class_count.argtypes = []
     lib.nfd_profile_class_name.argtypes = [C.c_int]
     lib.nfd_profile_class_name.restype = C.c_char_p
+    lib.nfd_attention_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                          vp, vp]
     lib.nfd_strerror.argtypes = [C.c_int]
     lib.nfd_strerror.restype = C.c_char_p
     _lib = lib
@@ -127,6 +129,27 @@ def accepted_frames(true_actions, i: int, k: int) -> int:
             break
         n += 1
     return n
+
+
+def attention_noalloc(q, k_pages, v_pages, n_q_frames: int, window: int, out, stream=None):
+    """nfd_attention_noalloc: block-causal attention without a context and without
+    any allocation (the caller passes `out`).  For hosts that may not call
+    cudaMalloc where they need attention (inside a stream capture, in a frame
+    loop that bans allocator calls, under a foreign memory arena).
+    q [H, n_q*T, dh]; k_pages, v_pages [n_kv, H, T, dh]; out [n_q*T, H*dh];
+    all on one device, same dtype (float32 or bfloat16), contiguous."""
+    lib = load()
+    n_kv, H, T, dh = k_pages.shape
+    dtype = I.DTYPE_BF16 if q.dtype == torch.bfloat16 else I.DTYPE_FP32
+    for t in (q, k_pages, v_pages, out):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == q.dtype
+    assert tuple(q.shape) == (H, n_q_frames * T, dh) and tuple(out.shape) == (n_q_frames * T, H * dh)
+    st = torch.cuda.current_stream(q.device) if stream is None else stream
+    _check(lib.nfd_attention_noalloc(C.c_void_p(q.data_ptr()), C.c_void_p(k_pages.data_ptr()),
+                                     C.c_void_p(v_pages.data_ptr()), dtype, H, dh, T, n_q_frames, n_kv, window,
+                                     C.c_void_p(out.data_ptr()), C.c_void_p(st.cuda_stream)),
+           "nfd_attention_noalloc")
+    return out
 
 
 class NFD:
