@@ -58,6 +58,7 @@ struct nfd_ctx {
     void *hbuf = nullptr, *qbuf = nullptr, *abuf = nullptr, *mbuf = nullptr;
     float *emb = nullptr, *h1 = nullptr, *sc = nullptr, *mod = nullptr, *fmod = nullptr;
     float *xp = nullptr, *vbuf = nullptr;       // sampler state, velocity
+    float2 *rope_cs = nullptr;                  // per-pass RoPE table [Nq_max][dh/2]
     StepParams *d_sp = nullptr;
     StepParams h_sp;
     unsigned long long *d_hash = nullptr;
@@ -265,6 +266,8 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
                (size_t)0);
     // tokens
     c->cls = CLS_PATCH;
+    if (c->bf16_mode && c->fast)
+        LAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, c->d_rope, c->rope_cs);
     LAUNCH(c, (k_patch_embed<TS>), M, 256, D.P * sizeof(float), sp, D, (const TS *)c->w_pe, (const TS *)c->b_pe,
            c->z);
     const int ln_grid = (M + 7) / 8;
@@ -272,7 +275,7 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
         const float *modl = c->mod + (size_t)l * 6 * d;
         c->cls = CLS_ADALN;
         LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0, (size_t)d);
-        EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l};
+        EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l, c->rope_cs};
         c->cls = CLS_GEMM_QKV;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV);
         if (kind == 1 && l == L - 1) break;      // a commit only needs the K/V of every layer
@@ -482,6 +485,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     A((void **)&c->d_hash, 8);
     A((void **)&c->d_status, 4);
     A((void **)&c->d_rope, sizeof(RopeTab));
+    A((void **)&c->rope_cs, Mmax * (D.dh / 2) * sizeof(float2));
     if (rc == NFD_OK) {
         std::vector<void *> v;
         v = c->w_mod; rc = upload_ptrs(c, v, &c->dp_wmod);

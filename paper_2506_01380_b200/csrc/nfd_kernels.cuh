@@ -134,8 +134,44 @@ __global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, con
 }
 
 // ---------------------------------------------------------------------------
-// GEMM epilogues.  Each is called with one output row m and two adjacent
-// columns (n, n+1), n even, holding the fp32 accumulators.
+// Per-pass RoPE table: (cos, sin) of every token's rotation angle for every
+// pair of the head dimension, [nf*T][dh/2].
+// ---------------------------------------------------------------------------
+__global__ void k_rope_table(const StepParams *sp, Dims D, const RopeTab *rt, float2 *tab) {
+    const int half = D.dh >> 1;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= sp->nf * D.T * half) return;
+    const int m = i / half, pi = i % half;
+    const int tok = m % D.T;
+    const int ax = rt->axis[pi];
+    const float pos = (float)(ax == 0 ? sp->fr[m / D.T].frame : (ax == 1 ? tok / D.tw : tok % D.tw));
+    float sn, cs;
+    sincosf(pos * rt->freq[pi], &sn, &cs);
+    tab[i] = make_float2(cs, sn);
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float *f) {
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 t = __bfloat1622float2(h[i]);
+        f[2 * i] = t.x;
+        f[2 * i + 1] = t.y;
+    }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float *f) {
+    uint4 u;
+    __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return u;
+}
+
+// ---------------------------------------------------------------------------
+// GEMM epilogues.  operator() takes one output row m and two adjacent columns
+// (n, n+1), n even, holding the fp32 accumulators (plain GEMM).  vec8() takes
+// eight adjacent columns n..n+7, n a multiple of 8 (tensor-core GEMM, bf16
+// storage only); it reads and writes 16 bytes at a time.
 // ---------------------------------------------------------------------------
 // QKV: + bias, 3D RoPE on q and k (Section 3.1 "3D Positional Embedding":
 // adjacent pairs, per-axis frequencies), q -> [H][Nq][dh], k/v -> cache pages.
@@ -146,6 +182,37 @@ template <typename TS> struct EpiQKV {
     const RopeTab *rt;
     Dims D;
     int layer;
+    const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by vec8
+    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+        float b[8];
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+        const int which = n / D.d, col = n - which * D.d;
+        const int head = col / D.dh, e = col - head * D.dh;
+        const int j = m / D.T, tok = m - j * D.T;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] += b[i];
+        TS *dst;
+        if (which < 2) {
+            const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
+            const float4 c01 = cs[0], c23 = cs[1];
+            const float cv[4] = {c01.x, c01.z, c23.x, c23.z}, sv[4] = {c01.y, c01.w, c23.y, c23.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float r0 = a[2 * i] * cv[i] - a[2 * i + 1] * sv[i];
+                const float r1 = a[2 * i] * sv[i] + a[2 * i + 1] * cv[i];
+                a[2 * i] = r0;
+                a[2 * i + 1] = r1;
+            }
+        }
+        if (which == 0) {
+            dst = q + ((size_t)head * (sp->nf * D.T) + m) * D.dh + e;
+        } else {
+            const FrameDesc fr = sp->fr[j];
+            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, fr.stream, layer, fr.frame) +
+                  ((size_t)head * D.T + tok) * D.dh + e;
+        }
+        *reinterpret_cast<uint4 *>(dst) = pack_bf16x8(a);
+    }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
         a0 += to_f(bias[n]);
         a1 += to_f(bias[n + 1]);
@@ -183,6 +250,25 @@ template <typename TS> struct EpiGateRes {
     const float *gate;      // mod + layer offset + chunk offset
     size_t row_stride;
     Dims D;
+    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+        float b[8];
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+        const int row = sp->fr[m / D.T].cond_row;
+        const float4 *g = reinterpret_cast<const float4 *>(gate + (size_t)row * row_stride + n);
+        float4 *zp = reinterpret_cast<float4 *>(z + (size_t)m * D.d + n);
+        const float4 g0 = g[0], g1 = g[1];
+        float4 z0 = zp[0], z1 = zp[1];
+        z0.x = fmaf(g0.x, a[0] + b[0], z0.x);
+        z0.y = fmaf(g0.y, a[1] + b[1], z0.y);
+        z0.z = fmaf(g0.z, a[2] + b[2], z0.z);
+        z0.w = fmaf(g0.w, a[3] + b[3], z0.w);
+        z1.x = fmaf(g1.x, a[4] + b[4], z1.x);
+        z1.y = fmaf(g1.y, a[5] + b[5], z1.y);
+        z1.z = fmaf(g1.z, a[6] + b[6], z1.z);
+        z1.w = fmaf(g1.w, a[7] + b[7], z1.w);
+        zp[0] = z0;
+        zp[1] = z1;
+    }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
         const int row = sp->fr[m / D.T].cond_row;
         const float *g = gate + (size_t)row * row_stride + n;
@@ -197,6 +283,13 @@ template <typename TS> struct EpiGelu {
     const TS *bias;
     TS *out;
     int N;
+    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+        float b[8];
+        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_f(a[i] + b[i]);
+        *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
+    }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
         TS *o = out + (size_t)m * N + n;
         o[0] = from_f<TS>(gelu_erf_f(a0 + to_f(bias[n])));
@@ -209,6 +302,10 @@ template <typename TS> struct EpiFinal {
     const StepParams *sp;
     const TS *bias;
     Dims D;
+    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) (*this)(m, n + i, a[i], a[i + 1]);
+    }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
         const int j = m / D.T, tok = m % D.T;
         const int r = tok / D.tw, c = tok % D.tw;
