@@ -226,10 +226,11 @@ template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int laye
     const Dims &D = c->D;
     c->cls = CLS_ATTN;
     prof_mark(c, false);
-    if (fast_attention<TS>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, D, nf, layer, (const TS *)c->qbuf,
-                           (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf)) {
+    const int n_fast = fast_attention<TS>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, D, nf, layer,
+                                          (const TS *)c->qbuf, (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
+    if (n_fast > 0) {
         prof_mark(c, true);
-        c->launches += fast_attention_launches();
+        c->launches += n_fast;
         return;
     }
     long long warps = (long long)nf * D.T * D.H;

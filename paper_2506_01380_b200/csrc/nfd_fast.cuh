@@ -7,6 +7,7 @@
 #include <tuple>
 
 #include "nfd_sm100.cuh"
+#include "nfd_attn_tc.cuh"
 
 enum { TC_NONE = 0, TC_QKV = 1, TC_RES = 2, TC_GELU = 3 };
 
@@ -20,6 +21,10 @@ struct FastState {
     int *d_status = nullptr;
     int n_sm = 148;
     size_t a_rows = 0;     // rows of every activation buffer (NFD_MAX_PASS_FRAMES * T)
+    AttnPlan plan;         // KB == 0: tensor-core attention not available for this shape
+    float *part_o = nullptr;
+    float2 *part_ml = nullptr;
+    size_t cache_rows = 0;
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;   // (ptr, rows, cols, box_rows)
 };
 
@@ -42,11 +47,33 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&fs.n_sm, cudaDevAttrMultiProcessorCount, dev);
     fs.ready = true;
+    // attention plan: head_dim 64, key blocks that divide the tokens per frame
+    AttnPlan pl;
+    const int KB = D.T % 128 == 0 ? 128 : (D.T % 112 == 0 ? 112 : (D.T % 64 == 0 ? 64 : 0));
+    fs.cache_rows = (size_t)D.n_streams * D.L * D.R * D.H * D.T;
+    if (D.dh == 64 && KB && D.H * D.T >= 128 && fs.cache_rows < 0x7fffffffull) {
+        pl.KB = KB;
+        pl.BPF = D.T / KB;
+        pl.QT = (D.T + 127) / 128;
+        const int target = fs.n_sm / (D.H * pl.QT) > 1 ? fs.n_sm / (D.H * pl.QT) : 1;
+        pl.CH = ((D.W + 1) * pl.BPF + target - 1) / target;
+        pl.MAXSPLIT = (D.R * pl.BPF + pl.CH - 1) / pl.CH;
+        const size_t items = (size_t)NFD_MAX_PASS_FRAMES * D.H * pl.QT * pl.MAXSPLIT * 128;
+        if (cudaMalloc((void **)&fs.part_o, items * 64 * sizeof(float)) != cudaSuccess ||
+            cudaMalloc((void **)&fs.part_ml, items * sizeof(float2)) != cudaSuccess) {
+            cudaGetLastError();
+            return NFD_E_NOMEM;
+        }
+        fs.plan = pl;
+    }
     return NFD_OK;
 }
 
 static void fast_destroy(FastState &fs) {
     fs.maps.clear();
+    if (fs.part_o) cudaFree(fs.part_o);
+    if (fs.part_ml) cudaFree(fs.part_ml);
+    fs.part_o = nullptr, fs.part_ml = nullptr;
     fs.ready = false;
 }
 
@@ -234,12 +261,41 @@ static bool fast_gemm(bool enabled, FastState &fs, cudaStream_t st, const StepPa
     }
 }
 
-static int fast_attention_launches() { return 1; }
+template <int KB>
+static int launch_attn_tc(FastState &fs, cudaStream_t st, const StepParams *sp, const Dims &D, int nf, int layer,
+                          const bf16 *q, const bf16 *kc, const bf16 *vc, bf16 *out) {
+    using A = AttnCfg<KB>;
+    static bool attr_set = false;
+    auto kern = k_attn_tc<KB>;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, A::SMEM) != cudaSuccess) {
+            cudaGetLastError();
+            return 0;
+        }
+        attr_set = true;
+    }
+    const CUtensorMap *mq = get_map_2d(fs, q, D.H * nf * D.T, 64, 128);
+    const CUtensorMap *mk = get_map_2d(fs, kc, (int)fs.cache_rows, 64, KB);
+    const CUtensorMap *mv = get_map_2d(fs, vc, (int)fs.cache_rows, 64, KB);
+    if (!mq || !mk || !mv) return 0;
+    const AttnPlan &pl = fs.plan;
+    dim3 grid(pl.MAXSPLIT, pl.QT, nf * D.H);
+    kern<<<grid, 192, A::SMEM, st>>>(*mq, *mk, *mv, sp, D, layer, pl, out, fs.part_o, fs.part_ml, fs.d_status);
+    if (pl.MAXSPLIT == 1) return 1;
+    k_attn_combine<<<dim3(pl.QT, nf * D.H), 128, 0, st>>>(sp, D, pl, fs.part_o, fs.part_ml, out);
+    return 2;
+}
 
+// Returns the number of kernels launched (0: not handled, use the plain kernel).
 template <typename TS>
-static bool fast_attention(bool enabled, FastState &fs, cudaStream_t st, const StepParams *sp, const Dims &D, int nf,
-                           int layer, const TS *q, const TS *kc, const TS *vc, TS *out) {
-    (void)enabled, (void)fs, (void)st, (void)sp, (void)D, (void)nf, (void)layer, (void)q, (void)kc, (void)vc,
-        (void)out;
-    return false;
+static int fast_attention(bool enabled, FastState &fs, cudaStream_t st, const StepParams *sp, const Dims &D, int nf,
+                          int layer, const TS *q, const TS *kc, const TS *vc, TS *out) {
+    if constexpr (!std::is_same<TS, bf16>::value) {
+        return 0;
+    } else {
+        if (!enabled || !fs.ready || fs.plan.KB == 0) return 0;
+        if (fs.plan.KB == 128) return launch_attn_tc<128>(fs, st, sp, D, nf, layer, q, kc, vc, out);
+        if (fs.plan.KB == 112) return launch_attn_tc<112>(fs, st, sp, D, nf, layer, q, kc, vc, out);
+        return launch_attn_tc<64>(fs, st, sp, D, nf, layer, q, kc, vc, out);
+    }
 }
