@@ -166,7 +166,7 @@ int nfd_kv_read(nfd_ctx *ctx, int stream, int layer, int frame, float *k_out, fl
  * storage type, [n_q_frames*T, n_heads*head_dim].  The data are first copied
  * into cache pages of batch slot 0 (which is reset), then the same attention
  * kernel the forward pass uses runs on them.
- * n_kv_frames <= W + k_max, n_q_frames <= k_max. */
+ * n_kv_frames <= W + k_max, n_q_frames <= k_max, window <= W. */
 int nfd_attention(nfd_ctx *ctx, const void *q, const void *k, const void *v, int n_q_frames, int n_kv_frames,
                   int window, void *out);
 

@@ -43,9 +43,11 @@ struct nfd_ctx {
     size_t esz = 4;
     bool use_graph = true, fast = true;
     long long launches = 0;
+    cudaError_t launch_err = cudaSuccess;    // first failed launch of the current pass
     std::vector<void *> allocs;
 
     // repacked weights: matrices [out][in], storage type
+    void *w_pe_io = nullptr;                    // patch embedding in its [P][d] layout
     void *w_pe = nullptr, *b_pe = nullptr, *w_t1 = nullptr, *b_t1 = nullptr, *w_t2 = nullptr, *b_t2 = nullptr;
     void *a_emb = nullptr, *w_fmod = nullptr, *b_fmod = nullptr, *w_out = nullptr, *b_out = nullptr;
     std::vector<void *> w_mod, b_mod, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2;
@@ -110,6 +112,7 @@ template <typename TS> static int repack_all(nfd_ctx *c, const nfd_weights *w) {
     const nfd_cfg &g = c->cfg;
     const int d = g.d_model, P = c->D.P, L = g.n_layers, dm = g.d_mlp;
     RET(repack_matrix<TS>(c, w->w_pe, P, d, &c->w_pe, true));
+    RET(repack_matrix<TS>(c, w->w_pe, P, d, &c->w_pe_io, false));
     RET(repack_matrix<TS>(c, w->b_pe, 1, d, &c->b_pe, false));
     RET(repack_matrix<TS>(c, w->w_t1, 256, d, &c->w_t1, true));
     RET(repack_matrix<TS>(c, w->b_t1, 1, d, &c->b_t1, false));
@@ -210,16 +213,31 @@ static void prof_mark(nfd_ctx *c, bool stop) {
         (c)->launches++;                                        \
     } while (0)
 
+// Kernels of a forward pass: launched with programmatic stream serialisation, so
+// that each one's prologue overlaps the tail of its predecessor.  Every such
+// kernel calls pdl_wait() before it touches global memory.
+#define PLAUNCH(c, kern, grid, block, smem, ...)                                                    \
+    do {                                                                                            \
+        prof_mark((c), false);                                                                      \
+        cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(block), (size_t)(smem), (c)->st, 1, __VA_ARGS__); \
+        if (le_ != cudaSuccess && !(c)->launch_err) (c)->launch_err = le_;                          \
+        prof_mark((c), true);                                                                       \
+        (c)->launches++;                                                                            \
+    } while (0)
+
 template <typename TS, typename Epi>
-static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind) {
+static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind,
+                        const void *next_w = nullptr, size_t next_elems = 0) {
     prof_mark(c, false);
-    if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, c->d_sp, c->D.T, A, Wt, M, N, K, epi, tc_kind)) {
+    // the next GEMM's weights, pulled towards L2 by this launch
+    const L2Prefetch pf{next_w, next_w ? (unsigned long long)(next_elems * sizeof(TS)) & ~15ull : 0ull};
+    if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, A, Wt, M, N, K, epi, tc_kind, pf)) {
         prof_mark(c, true);
         c->launches++;
         return;
     }
     dim3 grid((N + 63) / 64, (M + 63) / 64);
-    LAUNCH(c, (k_gemm_simple<TS, Epi>), grid, 256, 0, c->d_sp, c->D.T, A, Wt, N, K, epi);
+    PLAUNCH(c, (k_gemm_simple<TS, Epi>), grid, 256, 0, (const StepParams *)c->d_sp, c->D.T, A, Wt, N, K, epi);
 }
 
 template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int layer) {
@@ -236,14 +254,14 @@ template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int laye
     long long warps = (long long)nf * D.T * D.H;
     int grid = (int)((warps + 3) / 4);
     if (D.dh == 32)
-        LAUNCH(c, (k_attn_simple<TS, 32>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf, (const TS *)c->kc,
-               (const TS *)c->vc, (TS *)c->abuf);
+        PLAUNCH(c, (k_attn_simple<TS, 32>), grid, 128, 0, (const StepParams *)c->d_sp, D, layer, (const TS *)c->qbuf,
+                (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
     else if (D.dh == 64)
-        LAUNCH(c, (k_attn_simple<TS, 64>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf, (const TS *)c->kc,
-               (const TS *)c->vc, (TS *)c->abuf);
+        PLAUNCH(c, (k_attn_simple<TS, 64>), grid, 128, 0, (const StepParams *)c->d_sp, D, layer, (const TS *)c->qbuf,
+                (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
     else
-        LAUNCH(c, (k_attn_simple<TS, 128>), grid, 128, 0, c->d_sp, D, layer, (const TS *)c->qbuf,
-               (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
+        PLAUNCH(c, (k_attn_simple<TS, 128>), grid, 128, 0, (const StepParams *)c->d_sp, D, layer, (const TS *)c->qbuf,
+                (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
 }
 
 // Kernels after k_set_params.  nf and kind are fixed per captured graph.
@@ -254,50 +272,59 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     const size_t mod_row = (size_t)L * 6 * d;
     // conditioning
     c->cls = CLS_COND;
-    LAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
-    LAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
-           (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, c->emb, c->h1, 256, d, (size_t)d, (size_t)0);
-    LAUNCH(c, (k_gemv<TS, GEMV_T2>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t2,
-           (const TS *const *)(c->dp_t2 + 1), (const TS *)c->a_emb, c->h1, c->sc, d, d, (size_t)d, (size_t)0);
-    LAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((6 * d + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wmod,
-           (const TS *const *)c->dp_bmod, (const TS *)nullptr, c->sc, c->mod, d, 6 * d, mod_row, (size_t)6 * d);
+    PLAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
+    PLAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
+            (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, (const float *)c->emb, c->h1, 256, d, (size_t)d,
+            (size_t)0);
+    PLAUNCH(c, (k_gemv<TS, GEMV_T2>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t2,
+            (const TS *const *)(c->dp_t2 + 1), (const TS *)c->a_emb, (const float *)c->h1, c->sc, d, d, (size_t)d,
+            (size_t)0);
+    PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((6 * d + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wmod,
+            (const TS *const *)c->dp_bmod, (const TS *)nullptr, (const float *)c->sc, c->mod, d, 6 * d, mod_row,
+            (size_t)6 * d);
     if (kind == 0)
-        LAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((2 * d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_fmod,
-               (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, c->sc, c->fmod, d, 2 * d, (size_t)2 * d,
-               (size_t)0);
+        PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((2 * d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_fmod,
+                (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, (const float *)c->sc, c->fmod, d, 2 * d,
+                (size_t)2 * d, (size_t)0);
     // tokens
     c->cls = CLS_PATCH;
     if (c->bf16_mode && c->fast)
-        LAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, c->d_rope, c->rope_cs);
-    LAUNCH(c, (k_patch_embed<TS>), M, 256, D.P * sizeof(float), sp, D, (const TS *)c->w_pe, (const TS *)c->b_pe,
-           c->z);
-    const int ln_grid = (M + 7) / 8;
+        PLAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, (const RopeTab *)c->d_rope, c->rope_cs);
+    PLAUNCH(c, (k_patch_embed<TS>), (M + PE_TOK - 1) / PE_TOK, 256, PE_TOK * D.P * sizeof(float), sp, D,
+            (const TS *)c->w_pe_io, (const TS *)c->b_pe, c->z);
+    const int ln_grid = (M + 3) / 4;
     for (int l = 0; l < L; ++l) {
         const float *modl = c->mod + (size_t)l * 6 * d;
         c->cls = CLS_ADALN;
-        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0, (size_t)d);
-        EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l, c->rope_cs};
+        PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0,
+                (size_t)d);
+        EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l,
+                      c->rope_cs, M};
         c->cls = CLS_GEMM_QKV;
-        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV);
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV, c->w_o[l],
+                        (size_t)d * d);
         if (kind == 1 && l == L - 1) break;      // a commit only needs the K/V of every layer
         launch_attention<TS>(c, nf, l);
         EpiGateRes<TS> eo{sp, (const TS *)c->b_o[l], c->z, modl + 2 * d, mod_row, D};
         c->cls = CLS_GEMM_O;
-        launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES);
+        launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES, c->w_fc1[l],
+                        (size_t)d * D.dm);
         c->cls = CLS_ADALN;
-        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, modl, mod_row, (size_t)3 * d,
-               (size_t)4 * d);
+        PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row,
+                (size_t)3 * d, (size_t)4 * d);
         EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm};
         c->cls = CLS_GEMM_FC1;
-        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU);
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU, c->w_fc2[l],
+                        (size_t)d * D.dm);
         EpiGateRes<TS> e2{sp, (const TS *)c->b_fc2[l], c->z, modl + 5 * d, mod_row, D};
         c->cls = CLS_GEMM_FC2;
-        launch_gemm<TS>(c, (const TS *)c->mbuf, (const TS *)c->w_fc2[l], M, d, D.dm, e2, TC_RES);
+        launch_gemm<TS>(c, (const TS *)c->mbuf, (const TS *)c->w_fc2[l], M, d, D.dm, e2, TC_RES,
+                        l + 1 < L ? c->w_qkv[l + 1] : nullptr, (size_t)3 * d * d);
     }
     if (kind == 0) {
         c->cls = CLS_HEAD;
-        LAUNCH(c, (k_adaln<TS>), ln_grid, 256, 0, sp, D, c->z, (TS *)c->hbuf, c->fmod, (size_t)2 * d, (size_t)0,
-               (size_t)d);
+        PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, (const float *)c->fmod,
+                (size_t)2 * d, (size_t)0, (size_t)d);
         EpiFinal<TS> ef{sp, (const TS *)c->b_out, D};
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_out, M, D.P, d, ef, TC_NONE);
     }
@@ -315,9 +342,10 @@ static int run_pass(nfd_ctx *c) {
     const int nf = c->h_sp.nf, kind = c->h_sp.kind;
     if (!c->use_graph || c->st == nullptr || c->prof) {
         c->cls = CLS_PARAMS;
-        LAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
         enqueue_body_any(c, nf, kind);
         CK(cudaGetLastError());
+        CK(c->launch_err);
         return NFD_OK;
     }
     const int key = kind * 64 + nf + (c->fast ? 0 : 4096);
@@ -326,12 +354,14 @@ static int run_pass(nfd_ctx *c) {
         GraphEntry ge;
         long long before = c->launches;
         CK(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
-        LAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
         enqueue_body_any(c, nf, kind);
         cudaError_t e = cudaStreamEndCapture(c->st, &ge.graph);
         ge.launches = c->launches - before;
         c->launches = before;
+        if (e == cudaSuccess && c->launch_err != cudaSuccess) e = c->launch_err;
         if (e != cudaSuccess || !ge.graph) {
+            c->launch_err = cudaSuccess;
             fprintf(stderr, "libnfd: graph capture failed: %s\n", cudaGetErrorString(e));
             cudaGetLastError();
             return NFD_E_CUDA;
@@ -400,6 +430,7 @@ static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, 
             f.frame = c->n_total(streams[i]) + offset + j;
             f.win_first = f.frame - g.ctx_frames > 0 ? f.frame - g.ctx_frames : 0;
             f.cond_row = row;
+            f.first_new = c->n_total(streams[i]) + offset;
         }
     }
     p.nc = nc;
@@ -598,7 +629,7 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
     const int eg = (int)((ne + 255) / 256);
     // Section 4.1 "Sampling": start from pure noise at t' = pi/2
     c->cls = CLS_SAMPLER;
-    LAUNCH(c, k_axpby, eg, 256, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
+    PLAUNCH(c, k_axpby, eg, 256, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
     std::vector<float> tv(n);
     for (int s = 0; s < S; ++s) {
         const double tp = 0.5 * M_PI * (double)(S - s) / (double)S;
@@ -618,8 +649,8 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
             cn = cos(tpn), sn_next = sin(tpn) * sd;
         }
         c->cls = CLS_SAMPLER;
-        LAUNCH(c, k_sampler_post, eg, 256, 0, c->xp, c->vbuf, z, x0_out, (float)(sd * alpha), (float)(-sd * t),
-               (float)cn, (float)sn_next, ne);
+        PLAUNCH(c, k_sampler_post, eg, 256, 0, c->xp, (const float *)c->vbuf, z, x0_out, (float)(sd * alpha),
+                (float)(-sd * t), (float)cn, (float)sn_next, ne);
     }
     CK(cudaGetLastError());
     std::vector<int> fa((size_t)n * k);
@@ -703,7 +734,8 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
     if (!c || !q || !out) return NFD_E_NULLPTR;
     if ((k == nullptr) != (v == nullptr)) return NFD_E_NULLPTR;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return NFD_E_ALIGN;
-    if (n_q < 1 || n_q > c->cfg.max_spec || n_kv < n_q || n_kv > c->D.R || window < 0) return NFD_E_RANGE;
+    if (n_q < 1 || n_q > c->cfg.max_spec || n_kv < n_q || n_kv > c->D.R || window < 0 || window > c->D.W)
+        return NFD_E_RANGE;
     const Dims &D = c->D;
     c->n_committed[0] = 0;
     c->n_tentative[0] = 0;
@@ -729,9 +761,10 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
         p.fr[j].stream = 0;
         p.fr[j].frame = n_kv - n_q + j;
         p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
+        p.fr[j].first_new = n_kv - n_q;
     }
     c->cls = CLS_PARAMS;
-    LAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp);
+    PLAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp);
     if (c->bf16_mode)
         launch_attention<bf16>(c, n_q, 0);
     else
@@ -869,6 +902,7 @@ extern "C" int nfd_attention_noalloc(const void *q, const void *k_pages, const v
         p.fr[j].stream = 0;
         p.fr[j].frame = n_kv_frames - n_q_frames + j;
         p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
+        p.fr[j].first_new = n_kv_frames - n_q_frames;
     }
     // the descriptor is rewritten in full on every call; nothing of the previous call survives
     k_set_params<<<1, 256, 0, st>>>(p, d_sp);

@@ -6,15 +6,24 @@
 // block never straddles a page and the frame-granular mask needs no per-element
 // test at all).  Per block:
 //     S  = Q K^T          UMMA 128 x KB x 64, operands in shared memory (TMA),
-//                         accumulator in tensor memory (double buffered)
+//                         accumulator in tensor memory
 //     P  = exp2(S*c - m)  one thread per query row: TMEM -> registers, running
 //                         max / sum, bf16 P written to shared memory
-//     PV = P V            UMMA 128 x 64 x KB, V used straight from its page
-//                         (MN-major B operand), accumulator in tensor memory
-//     O  = O*corr + PV    in registers
-// Warp 0 = TMA producer, warp 1 = UMMA issuer, warps 2-5 = softmax.
-// A key range longer than CH blocks is split over several CTAs which write
-// unnormalised (O, m, l) partials; k_attn_combine merges them in split order.
+//     O += P V            UMMA 128 x 64 x KB, V used straight from its page
+//                         (MN-major B operand), accumulated in tensor memory
+// The reference maximum m of a row is raised only when a block's maximum exceeds
+// it by more than 2^8; only then is the row's O accumulator rescaled (in tensor
+// memory), so that in the steady state O is never read back.  The final
+// normalisation by the running sum makes the result independent of that choice.
+// Warp 0 = TMA producer, warp 1 = UMMA issuer, warps 2-5 and 6-9 = two softmax
+// groups.  Group g takes the key blocks b with b % 2 == g and keeps its own
+// (max, sum, O) state, S accumulator and P tile, so that one group's
+// exponentials overlap the other's tensor-memory traffic and UMMAs.
+// A key range longer than CH blocks is split over several CTAs; every group of
+// every split writes its unnormalised (O, m, l) state, and the CTA that finishes
+// last (a counter per query tile) merges all states in (split, group) order and
+// writes the output.  With a single split the two groups are merged in shared
+// memory instead.
 // CH depends only on the configuration, so a frame's result does not depend on
 // which other frames share its pass.
 #pragma once
@@ -31,10 +40,15 @@ struct AttnPlan {
 template <int KB> struct AttnCfg {
     static constexpr int NST = 4;                          // K/V ring stages
     static constexpr int Q_BYTES = 128 * 128;
-    static constexpr int P_BYTES = 2 * 128 * 128;          // two 64-key atoms
+    static constexpr int P_BYTES = 2 * 128 * 128;          // one group's P tile: two 64-key atoms
     static constexpr int KV_BYTES = KB * 128;              // one K (or V) block
-    static constexpr int SMEM = Q_BYTES + P_BYTES + NST * 2 * KV_BYTES + 1024 + 256;
-    static constexpr int TMEM_COLS = 512;                  // S0 @0, S1 @128, PV @256
+    static constexpr int RING_BYTES = NST * 2 * KV_BYTES;
+    static constexpr int OROW = 68;                        // floats per parked O row (64 + pad)
+    static constexpr int PARK_BYTES = 128 * OROW * 4 + 128 * 8;           // group 1's state: O rows, then (m, l)
+    static constexpr int SMEM = Q_BYTES + 2 * P_BYTES + RING_BYTES + 1024 + 256;
+    static constexpr int TMEM_COLS = 512;                  // S0 @0, S1 @128, O0 @256, O1 @320
+    static constexpr int THREADS = 320;
+    static_assert(PARK_BYTES <= 2 * P_BYTES, "group 1's parked state must fit the P tiles");
 };
 
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_bmn(int M, int N) {
@@ -47,48 +61,55 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+__device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
 template <int KB>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(AttnCfg<KB>::THREADS, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
           const __grid_constant__ CUtensorMap tmV, const StepParams *sp, Dims D, int layer, AttnPlan pl, bf16 *out,
-          float *part_o, float2 *part_ml, int *status) {
+          float *part_o, float2 *part_ml, unsigned int *counters, int *status) {
     using A = AttnCfg<KB>;
     extern __shared__ uint8_t smem_raw[];
     const int z = blockIdx.z, j = z / D.H, h = z % D.H;
     const int qt = blockIdx.y, split = blockIdx.x;
+    // the pass descriptor was written by the first kernel of the pass, which completed long ago
     const FrameDesc fr = sp->fr[j];
     const int nbt = (fr.frame - fr.win_first + 1) * pl.BPF;      // key blocks of this frame's window
     const int nsplit = (nbt + pl.CH - 1) / pl.CH;
-    if (split >= nsplit) return;                                  // uniform for the CTA
+    if (split >= nsplit) return;                                  // uniform for the CTA, before any barrier or allocation
     const int b0 = split * pl.CH;
-    const int nb = min(nbt, b0 + pl.CH) - b0;
+    const int nb = min(nbt, b0 + pl.CH) - b0;                     // >= 1
     const int Nq = sp->nf * D.T;
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *sQ = smem, *sP = smem + A::Q_BYTES, *sKV = sP + A::P_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + A::NST * 2 * A::KV_BYTES);
+    uint8_t *sQ = smem, *sP = smem + A::Q_BYTES, *sKV = sP + 2 * A::P_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + A::RING_BYTES);
     const uint32_t q_full = smem_u32(bars), kv_full = smem_u32(bars + 1), kv_empty = smem_u32(bars + 1 + A::NST),
-                   s_full = smem_u32(bars + 1 + 2 * A::NST), s_empty = s_full + 16, p_full = s_full + 32,
-                   pv_full = s_full + 40;
+                   s_full = smem_u32(bars + 1 + 2 * A::NST), p_full = s_full + 16, pv_done = s_full + 32;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 1 + 2 * A::NST + 6);
+    int *last_flag = reinterpret_cast<int *>(tmem_slot + 1);
+    // group 1 parks its state here after the main loop (the P tiles are free by then)
+    float *parkO = reinterpret_cast<float *>(sP);
+    float2 *parkML = reinterpret_cast<float2 *>(sP + 128 * A::OROW * 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
         mbar_init(q_full, 1);
         for (int s = 0; s < A::NST; ++s) {
             mbar_init(kv_full + 8 * s, 1);
             mbar_init(kv_empty + 8 * s, 1);
         }
-        mbar_init(s_full, 1);
-        mbar_init(s_full + 8, 1);
-        mbar_init(s_empty, 128);
-        mbar_init(s_empty + 8, 128);
-        mbar_init(p_full, 128);
-        mbar_init(pv_full, 1);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(s_full + 8 * g, 1);
+            mbar_init(p_full + 8 * g, 128);
+            mbar_init(pv_done + 8 * g, 1);
+        }
         fence_mbar_init();
-        tma_prefetch_desc(&tmQ);
-        tma_prefetch_desc(&tmK);
-        tma_prefetch_desc(&tmV);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), A::TMEM_COLS);
@@ -98,217 +119,288 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tS0 = tmem, tPV = tmem + 256;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            mbar_expect_tx(q_full, A::Q_BYTES);
-            tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
             const int page_rows = D.H * D.T;
+            bool waited = false;
             for (int b = 0; b < nb; ++b) {
                 const int s = b % A::NST;
-                if (b >= A::NST && !mbar_wait(kv_empty + 8 * s, ((b / A::NST) - 1) & 1, status)) break;
                 const int blk = b0 + b;
                 const int g = fr.win_first + blk / pl.BPF, kb = blk % pl.BPF;
+                // pages of frames written earlier than this pass may be fetched before the predecessor finishes
+                if (!waited && (g >= fr.first_new || b >= A::NST)) {
+                    pdl_wait();
+                    waited = true;
+                    mbar_expect_tx(q_full, A::Q_BYTES);
+                    tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
+                }
+                if (b >= A::NST && !mbar_wait(kv_empty + 8 * s, ((b / A::NST) - 1) & 1, status)) break;
                 const int row = ((fr.stream * D.L + layer) * D.R + (g % D.R)) * page_rows + h * D.T + kb * KB;
                 mbar_expect_tx(kv_full + 8 * s, 2 * A::KV_BYTES);
                 tma_load_2d(smem_u32(sKV + s * 2 * A::KV_BYTES), &tmK, kv_full + 8 * s, 0, row);
                 tma_load_2d(smem_u32(sKV + s * 2 * A::KV_BYTES + A::KV_BYTES), &tmV, kv_full + 8 * s, 0, row);
             }
+            if (!waited) {
+                pdl_wait();
+                mbar_expect_tx(q_full, A::Q_BYTES);
+                tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
+            }
         }
     } else if (warp == 1) {
         // ---------------- UMMA issuer ----------------
         if (lane == 0) {
+            pdl_launch();
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, KB);
             constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(128, 64);
             const uint64_t qd = umma_desc_k128(smem_u32(sQ));
-            const uint64_t pd = umma_desc_k128(smem_u32(sP));
-            bool ok = mbar_wait(q_full, 0, status) && mbar_wait(kv_full, 0, status);
-            if (ok) {
+            bool ok = mbar_wait(q_full, 0, status);
+            auto issue_s = [&](int b) {          // S(b) = Q K(b)^T into group (b & 1)'s accumulator
+                const int s = b % A::NST, g = b & 1;
+                if (!mbar_wait(kv_full + 8 * s, (b / A::NST) & 1, status)) return false;
                 tc_fence_after();
-                const uint64_t kd = umma_desc_k128(smem_u32(sKV));
+                const uint64_t kd = umma_desc_k128(smem_u32(sKV + s * 2 * A::KV_BYTES));
 #pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4) umma_bf16_ss(tS0, qd + 2 * k4, kd + 2 * k4, idesc_s, k4 != 0);
-                umma_commit(s_full);
-            }
+                for (int k4 = 0; k4 < 4; ++k4) umma_bf16_ss(tmem + 128 * g, qd + 2 * k4, kd + 2 * k4, idesc_s, k4 != 0);
+                umma_commit(s_full + 8 * g);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            if (ok && nb > 1) ok = issue_s(1);
             for (int b = 0; b < nb && ok; ++b) {
-                if (b + 1 < nb) {
-                    const int b1 = b + 1, s1 = b1 % A::NST;
-                    ok = mbar_wait(kv_full + 8 * s1, (b1 / A::NST) & 1, status);
-                    if (ok && b1 >= 2) ok = mbar_wait(s_empty + 8 * (b1 & 1), ((b1 >> 1) - 1) & 1, status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint64_t kd = umma_desc_k128(smem_u32(sKV + s1 * 2 * A::KV_BYTES));
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        umma_bf16_ss(tS0 + 128 * (b1 & 1), qd + 2 * k4, kd + 2 * k4, idesc_s, k4 != 0);
-                    umma_commit(s_full + 8 * (b1 & 1));
-                }
-                ok = mbar_wait(p_full, b & 1, status);
+                const int g = b & 1, s = b % A::NST;
+                ok = mbar_wait(p_full + 8 * g, (b >> 1) & 1, status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t vd = umma_desc_k128(smem_u32(sKV + (b % A::NST) * 2 * A::KV_BYTES + A::KV_BYTES));
+                const uint64_t pd = umma_desc_k128(smem_u32(sP + g * A::P_BYTES));
+                const uint64_t vd = umma_desc_k128(smem_u32(sKV + s * 2 * A::KV_BYTES + A::KV_BYTES));
 #pragma unroll
                 for (int i = 0; i < KB / 16; ++i) {
                     // P: K-major, 64-key atoms of 16 KiB; V: MN-major, 16 keys = 2 KiB per step
                     const uint64_t pa = pd + (uint64_t)((i >> 2) * (16384 >> 4) + (i & 3) * 2);
-                    umma_bf16_ss(tPV, pa, vd + (uint64_t)(i * (2048 >> 4)), idesc_pv, i != 0);
+                    umma_bf16_ss(tmem + 256 + 64 * g, pa, vd + (uint64_t)(i * (2048 >> 4)), idesc_pv,
+                                 (uint32_t)((b >> 1) != 0 || i != 0));
                 }
-                umma_commit(pv_full);
-                umma_commit(kv_empty + 8 * (b % A::NST));
+                umma_commit(pv_done + 8 * g);
+                umma_commit(kv_empty + 8 * s);
+                if (b + 2 < nb) ok = issue_s(b + 2);
             }
         }
     } else {
-        // ---------------- softmax: one thread per query row ----------------
+        // ---------------- softmax: one thread per query row, two groups ----------------
+        const int g = (warp - 2) >> 2;                     // group: blocks b with (b & 1) == g
         const int quad = warp & 3;
         const int trow = quad * 32 + lane;
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+        const uint32_t tS = tmem + 128 * g + lane_off, tO = tmem + 256 + 64 * g + lane_off;
         const float c = (1.0f / sqrtf((float)D.dh)) * 1.4426950408889634f;   // softmax scale in the log2 domain
         float m_run = -INFINITY, l_run = 0.f;
+        uint8_t *prow = sP + g * A::P_BYTES + trow * 128;
+        bool ok = true;
+        int i = 0;
+        for (int b = g; b < nb; b += 2, ++i) {
+            ok = mbar_wait(s_full + 8 * g, i & 1, status);
+            if (!ok) break;
+            tc_fence_after();
+            // pass 1 over S: row maximum (all loads in flight together; the values die right after)
+            float mx;
+            {
+                uint32_t sr[KB];
+#pragma unroll
+                for (int cc = 0; cc < KB; cc += 32) {
+                    if (cc + 32 <= KB)
+                        tmem_ld32(tS + cc, sr + cc);
+                    else
+                        tmem_ld16(tS + cc, sr + cc);
+                }
+                tmem_ld_wait();
+                float m4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]),
+                               __uint_as_float(sr[3])};
+#pragma unroll
+                for (int e = 4; e < KB; ++e) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(sr[e]));
+                mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            }
+            const float m_blk = mx * c;
+            if (i > 0) {
+                // the previous P V product of this group is complete: its P tile is free, O is at rest
+                ok = mbar_wait(pv_done + 8 * g, (i - 1) & 1, status);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            const bool raise = m_blk > m_run + 8.0f;       // always true for the first block (m_run = -inf)
+            if (__any_sync(0xffffffffu, raise)) {
+                const float m_new = raise ? m_blk : m_run;
+                const float f = ex2_approx(m_run - m_new);  // 1 for rows that keep their reference maximum
+                if (i > 0) {
+#pragma unroll
+                    for (int cc = 0; cc < 64; cc += 32) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + cc, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+                        tmem_st32(tO + cc, r);
+                    }
+                    tmem_st_wait();
+                }
+                l_run *= f;
+                m_run = m_new;
+            }
+            // pass 2 over S, 16 columns at a time with the next load in flight:
+            // P = exp2(S c - m) as bf16 into shared memory (128-byte-swizzled K-major layout)
+            float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t sa[16], sb[16];
+            tmem_ld16(tS, sa);
+#pragma unroll
+            for (int cc = 0; cc < KB; cc += 16) {
+                uint32_t *cur = ((cc >> 4) & 1) ? sb : sa, *nxt = ((cc >> 4) & 1) ? sa : sb;
+                tmem_ld_wait();
+                if (cc + 16 < KB) tmem_ld16(tS + cc + 16, nxt);
+#pragma unroll
+                for (int u2 = 0; u2 < 2; ++u2) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(cur[8 * u2 + 2 * u]), c, -m_run));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(cur[8 * u2 + 2 * u + 1]), c, -m_run));
+                        ls4[u] += p0 + p1;
+                        const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
+                        pk[u] = *reinterpret_cast<const uint32_t *>(&hp);
+                    }
+                    const int ch = (cc >> 3) + u2;
+                    uint8_t *dst = prow + (ch >> 3) * 16384 + (((ch & 7) ^ (trow & 7)) << 4);
+                    *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(p_full + 8 * g);
+        }
+        // this group's O accumulator (unnormalised, relative to m_run)
         float O[64];
 #pragma unroll
         for (int e = 0; e < 64; ++e) O[e] = 0.f;
-        uint8_t *prow = sP + trow * 128;
-        bool ok = true;
-        for (int b = 0; b < nb; ++b) {
-            ok = mbar_wait(s_full + 8 * (b & 1), (b >> 1) & 1, status);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t sr[KB];
-            const uint32_t ts = tS0 + 128 * (b & 1) + lane_off;
-#pragma unroll
-            for (int cc = 0; cc < KB; cc += 32) {
-                if (cc + 32 <= KB)
-                    tmem_ld32(ts + cc, sr + cc);
-                else
-                    tmem_ld16(ts + cc, sr + cc);
-            }
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(s_empty + 8 * (b & 1));
-            float mx = __uint_as_float(sr[0]);
-#pragma unroll
-            for (int i = 1; i < KB; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
-            const float m_new = fmaxf(m_run, mx * c);
-            const float corr = ex2_approx(m_run - m_new);
-            float ls = 0.f;
-            uint32_t pk[KB / 2];
-#pragma unroll
-            for (int i = 0; i < KB; i += 2) {
-                const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i]), c, -m_new));
-                const float p1 = ex2_approx(fmaf(__uint_as_float(sr[i + 1]), c, -m_new));
-                // the row sum uses the bf16-rounded probabilities that the P V product sees
-                const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
-                const float2 pf = __bfloat1622float2(hp);
-                ls += pf.x + pf.y;
-                pk[i >> 1] = *reinterpret_cast<const uint32_t *>(&hp);
-            }
-            l_run = fmaf(l_run, corr, ls);
-            m_run = m_new;
-            if (b > 0) {
-                ok = mbar_wait(pv_full, (b - 1) & 1, status);
-                if (!ok) break;
-                tc_fence_after();
-#pragma unroll
-                for (int cc = 0; cc < 64; cc += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tPV + lane_off + cc, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) O[cc + e] += __uint_as_float(r[e]);
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < 64; ++e) O[e] *= corr;
-            // P (bf16) into shared memory in the 128-byte-swizzled K-major layout
-#pragma unroll
-            for (int ch = 0; ch < KB / 8; ++ch) {
-                uint8_t *dst = prow + (ch >> 3) * 16384 + (((ch & 7) ^ (trow & 7)) << 4);
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-            }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            mbar_arrive(p_full);
-        }
-        if (ok && nb > 0) {
-            ok = mbar_wait(pv_full, (nb - 1) & 1, status);
+        if (ok && i > 0) {
+            ok = mbar_wait(pv_done + 8 * g, (i - 1) & 1, status);
             if (ok) {
                 tc_fence_after();
 #pragma unroll
                 for (int cc = 0; cc < 64; cc += 32) {
                     uint32_t r[32];
-                    tmem_ld32(tPV + lane_off + cc, r);
+                    tmem_ld32(tO + cc, r);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) O[cc + e] += __uint_as_float(r[e]);
+                    for (int e = 0; e < 32; ++e) O[cc + e] = __uint_as_float(r[e]);
                 }
             }
         }
+        if (!ok || i == 0) {                               // no block or a failed wait: this state counts for nothing
+            m_run = -INFINITY, l_run = 0.f;
+#pragma unroll
+            for (int e = 0; e < 64; ++e) O[e] = 0.f;
+        }
         const int row = qt * 128 + trow;
-        if (ok && row < D.T) {
-            if (nsplit == 1) {
-                const float inv = 1.0f / l_run;
+        const size_t item_q = (size_t)z * pl.QT + qt;      // (frame, head, query tile)
+        if (nsplit == 1) {
+            // ---- one CTA holds the whole window: group 1 parks its state, group 0 folds it in ----
+            named_bar_sync(1, 256);                        // both groups are past their last UMMA: the P tiles are free
+            if (g == 1) {
+                float4 *po = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);
+#pragma unroll
+                for (int e = 0; e < 64; e += 4) po[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
+                parkML[trow] = make_float2(m_run, l_run);
+            }
+            named_bar_sync(1, 256);
+            if (g == 0 && row < D.T) {
+                const float2 ml1 = parkML[trow];
+                const float m = fmaxf(m_run, ml1.x);
+                const float w0 = ex2_approx(m_run - m), w1 = ex2_approx(ml1.x - m);
+                const float inv = 1.0f / (l_run * w0 + ml1.y * w1);
+                const float a0 = w0 * inv, a1 = w1 * inv;
+                const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)trow * A::OROW);
                 bf16 *o = out + (size_t)(j * D.T + row) * D.d + h * 64;
 #pragma unroll
                 for (int e = 0; e < 64; e += 8) {
-                    float t[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) t[u] = O[e + u] * inv;
+                    const float4 v0 = po[e >> 2], v1 = po[(e >> 2) + 1];
+                    float t[8] = {fmaf(O[e], a0, v0.x * a1),     fmaf(O[e + 1], a0, v0.y * a1),
+                                  fmaf(O[e + 2], a0, v0.z * a1), fmaf(O[e + 3], a0, v0.w * a1),
+                                  fmaf(O[e + 4], a0, v1.x * a1), fmaf(O[e + 5], a0, v1.y * a1),
+                                  fmaf(O[e + 6], a0, v1.z * a1), fmaf(O[e + 7], a0, v1.w * a1)};
                     *reinterpret_cast<uint4 *>(o + e) = pack_bf16x8(t);
                 }
-            } else {
-                const size_t item = ((size_t)(z * pl.QT + qt) * pl.MAXSPLIT + split) * 128 + trow;
-                float4 *po = reinterpret_cast<float4 *>(part_o + item * 64);
+            }
+        } else {
+            // ---- both groups publish their state; the CTA that finishes last merges all 2*nsplit states ----
+            const size_t st0 = item_q * (2 * pl.MAXSPLIT) * 128;                     // first state row of this query tile
+            {
+                const size_t item = st0 + (size_t)(2 * split + g) * 128 + trow;
+                float4 *po4 = reinterpret_cast<float4 *>(part_o + item * 64);
 #pragma unroll
-                for (int e = 0; e < 64; e += 4) po[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
+                for (int e = 0; e < 64; e += 4) po4[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
                 part_ml[item] = make_float2(m_run, l_run);
+            }
+            __threadfence();
+            named_bar_sync(1, 256);
+            if (threadIdx.x == 64) {
+                const unsigned int prev = atomicAdd(counters + item_q, 1u);
+                const int last = prev == (unsigned int)(nsplit - 1);
+                if (last) counters[item_q] = 0;            // ready for the next launch
+                *last_flag = last;
+            }
+            named_bar_sync(1, 256);
+            if (*last_flag) {
+                __threadfence();
+                const int ns = 2 * nsplit;                 // states, in (split, group) order
+                for (int it = (int)threadIdx.x - 64; it < 128 * 8; it += 256) {
+                    const int r = it >> 3, ch = it & 7;
+                    const int orow = qt * 128 + r;
+                    if (orow >= D.T) continue;
+                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    float l = 0.f, mx = -INFINITY;
+                    for (int s0 = 0; s0 < ns; s0 += 6) {
+                        // six states at a time, all loads in flight together
+                        float2 ml[6];
+                        float4 v0[6], v1[6];
+#pragma unroll
+                        for (int u = 0; u < 6; ++u) {
+                            const int s = s0 + u < ns ? s0 + u : ns - 1;
+                            const size_t item = st0 + (size_t)s * 128 + r;
+                            ml[u] = __ldcg(&part_ml[item]);
+                            const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch * 8);
+                            v0[u] = __ldcg(po), v1[u] = __ldcg(po + 1);
+                        }
+                        float mb = mx;
+#pragma unroll
+                        for (int u = 0; u < 6; ++u)
+                            if (s0 + u < ns) mb = fmaxf(mb, ml[u].x);
+                        const float fo = ex2_approx(mx - mb);          // rescale of what was merged so far (0 at first)
+                        l *= fo;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[e] *= fo;
+                        mx = mb;
+#pragma unroll
+                        for (int u = 0; u < 6; ++u) {
+                            if (s0 + u < ns) {
+                                const float w = ex2_approx(ml[u].x - mx);
+                                l = fmaf(ml[u].y, w, l);
+                                acc[0] = fmaf(v0[u].x, w, acc[0]), acc[1] = fmaf(v0[u].y, w, acc[1]);
+                                acc[2] = fmaf(v0[u].z, w, acc[2]), acc[3] = fmaf(v0[u].w, w, acc[3]);
+                                acc[4] = fmaf(v1[u].x, w, acc[4]), acc[5] = fmaf(v1[u].y, w, acc[5]);
+                                acc[6] = fmaf(v1[u].z, w, acc[6]), acc[7] = fmaf(v1[u].w, w, acc[7]);
+                            }
+                        }
+                    }
+                    const float inv = 1.0f / l;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) acc[u] *= inv;
+                    *reinterpret_cast<uint4 *>(out + (size_t)(j * D.T + orow) * D.d + h * 64 + ch * 8) = pack_bf16x8(acc);
+                }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, A::TMEM_COLS);
-}
-
-// Merge the split partials of one (frame, head, query tile): thread = query row.
-__global__ void __launch_bounds__(128) k_attn_combine(const StepParams *sp, Dims D, AttnPlan pl, const float *part_o,
-                                                      const float2 *part_ml, bf16 *out) {
-    const int z = blockIdx.y, j = z / D.H, h = z % D.H, qt = blockIdx.x;
-    const FrameDesc fr = sp->fr[j];
-    const int nbt = (fr.frame - fr.win_first + 1) * pl.BPF;
-    const int nsplit = (nbt + pl.CH - 1) / pl.CH;
-    if (nsplit == 1) return;                      // the attention kernel already wrote the result
-    const int trow = threadIdx.x, row = qt * 128 + trow;
-    if (row >= D.T) return;
-    const size_t item0 = ((size_t)(z * pl.QT + qt) * pl.MAXSPLIT) * 128 + trow;
-    float mx = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) mx = fmaxf(mx, part_ml[item0 + (size_t)s * 128].x);
-    float acc[64];
-#pragma unroll
-    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
-    float l = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-        const float2 ml = part_ml[item0 + (size_t)s * 128];
-        const float w = ex2_approx(ml.x - mx);
-        l = fmaf(ml.y, w, l);
-        const float4 *po = reinterpret_cast<const float4 *>(part_o + (item0 + (size_t)s * 128) * 64);
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-            const float4 v = po[e];
-            acc[4 * e] = fmaf(v.x, w, acc[4 * e]);
-            acc[4 * e + 1] = fmaf(v.y, w, acc[4 * e + 1]);
-            acc[4 * e + 2] = fmaf(v.z, w, acc[4 * e + 2]);
-            acc[4 * e + 3] = fmaf(v.w, w, acc[4 * e + 3]);
-        }
-    }
-    const float inv = 1.0f / l;
-    bf16 *o = out + (size_t)(j * D.T + row) * D.d + h * 64;
-#pragma unroll
-    for (int e = 0; e < 64; e += 8) {
-        float t[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) t[u] = acc[e + u] * inv;
-        *reinterpret_cast<uint4 *>(o + e) = pack_bf16x8(t);
-    }
 }

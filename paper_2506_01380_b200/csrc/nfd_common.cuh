@@ -13,6 +13,7 @@ struct FrameDesc {
     int frame;       // absolute frame index (RoPE position, ring slot = frame % R)
     int win_first;   // first frame this one attends to (>= 0, >= frame - W)
     int cond_row;    // row of the conditioning / modulation tables
+    int first_new;   // first frame of this stream whose K/V the current pass writes (earlier pages are final)
 };
 
 // One distinct (FM time, action) pair of a pass.
@@ -55,6 +56,16 @@ struct RopeTab {
     int axis[NFD_MAX_HALF_DH];
 };
 
+// ---- programmatic dependent launch ------------------------------------------
+// Every kernel of a pass is launched with programmatic stream serialisation: it
+// may start while its predecessor is still running.  pdl_wait() blocks until the
+// predecessor grids have completed and their writes are visible; anything that
+// does not depend on them (barrier set-up, tensor-memory allocation, weight
+// prefetch) goes before it.  pdl_launch() lets the successor start its own
+// prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
@@ -68,6 +79,21 @@ __device__ __forceinline__ size_t kv_page_offset(const Dims &D, int stream, int 
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+
+// GELU (erf form) for values that are rounded to bf16 afterwards: erf by the
+// rational approximation 7.1.26 of Abramowitz & Stegun (absolute error below
+// 1.5e-7, three orders of magnitude under the bf16 rounding step).
+__device__ __forceinline__ float gelu_erf_bf16_f(float x) {
+    const float ax = fabsf(x);
+    const float z = ax * 0.70710678118654752440f;
+    const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+    float p = fmaf(1.061405429f, t, -1.453152027f);
+    p = fmaf(p, t, 1.421413741f);
+    p = fmaf(p, t, -0.284496736f);
+    p = fmaf(p, t, 0.254829592f);
+    const float e = fmaf(-p * t, __expf(-z * z), 1.0f);      // erf(|x|/sqrt 2)
+    return 0.5f * fmaf(ax, e, x);                            // x/2 (1 + sign(x) e)
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -5,8 +5,10 @@
 #pragma once
 #include <map>
 #include <tuple>
+#include <utility>
 
 #include "nfd_sm100.cuh"
+#include "nfd_gemm_tc.cuh"
 #include "nfd_attn_tc.cuh"
 
 enum { TC_NONE = 0, TC_QKV = 1, TC_RES = 2, TC_GELU = 3 };
@@ -22,8 +24,9 @@ struct FastState {
     int n_sm = 148;
     size_t a_rows = 0;     // rows of every activation buffer (NFD_MAX_PASS_FRAMES * T)
     AttnPlan plan;         // KB == 0: tensor-core attention not available for this shape
-    float *part_o = nullptr;
+    float *part_o = nullptr;           // per (split, softmax group) states of the attention kernel
     float2 *part_ml = nullptr;
+    unsigned int *attn_counters = nullptr;   // one per (frame, head, query tile); zero between launches
     size_t cache_rows = 0;
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;   // (ptr, rows, cols, box_rows)
 };
@@ -55,14 +58,21 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
         pl.KB = KB;
         pl.BPF = D.T / KB;
         pl.QT = (D.T + 127) / 128;
+        // split the longest window (a frame sees at most W + 1 pages) so that heads x query tiles x splits
+        // fills the SMs once
         const int target = fs.n_sm / (D.H * pl.QT) > 1 ? fs.n_sm / (D.H * pl.QT) : 1;
         pl.CH = ((D.W + 1) * pl.BPF + target - 1) / target;
-        pl.MAXSPLIT = (D.R * pl.BPF + pl.CH - 1) / pl.CH;
-        const size_t items = (size_t)NFD_MAX_PASS_FRAMES * D.H * pl.QT * pl.MAXSPLIT * 128;
-        if (cudaMalloc((void **)&fs.part_o, items * 64 * sizeof(float)) != cudaSuccess ||
-            cudaMalloc((void **)&fs.part_ml, items * sizeof(float2)) != cudaSuccess) {
-            cudaGetLastError();
-            return NFD_E_NOMEM;
+        pl.MAXSPLIT = ((D.W + 1) * pl.BPF + pl.CH - 1) / pl.CH;
+        if (pl.MAXSPLIT > 1) {
+            const size_t tiles = (size_t)NFD_MAX_PASS_FRAMES * D.H * pl.QT;
+            const size_t items = tiles * 2 * pl.MAXSPLIT * 128;      // one state per (split, softmax group)
+            if (cudaMalloc((void **)&fs.part_o, items * 64 * sizeof(float)) != cudaSuccess ||
+                cudaMalloc((void **)&fs.part_ml, items * sizeof(float2)) != cudaSuccess ||
+                cudaMalloc((void **)&fs.attn_counters, tiles * sizeof(unsigned int)) != cudaSuccess ||
+                cudaMemset(fs.attn_counters, 0, tiles * sizeof(unsigned int)) != cudaSuccess) {
+                cudaGetLastError();
+                return NFD_E_NOMEM;
+            }
         }
         fs.plan = pl;
     }
@@ -73,7 +83,8 @@ static void fast_destroy(FastState &fs) {
     fs.maps.clear();
     if (fs.part_o) cudaFree(fs.part_o);
     if (fs.part_ml) cudaFree(fs.part_ml);
-    fs.part_o = nullptr, fs.part_ml = nullptr;
+    if (fs.attn_counters) cudaFree(fs.attn_counters);
+    fs.part_o = nullptr, fs.part_ml = nullptr, fs.attn_counters = nullptr;
     fs.ready = false;
 }
 
@@ -99,130 +110,81 @@ static const CUtensorMap *get_map_2d(FastState &fs, const void *ptr, int rows, i
 }
 
 // ---------------------------------------------------------------------------
-// C[M,N] = A[M,K] * Wt[N,K]^T, bf16 in, fp32 accumulation in tensor memory.
-// One CTA per 128 x BN output tile.  Warp 0: TMA producer; warp 1: TMEM
-// allocation and UMMA issue; warps 2-5: epilogue (TMEM -> registers -> fused
-// epilogue functor).  K is walked in 64-element blocks through a STAGES-deep
-// shared-memory ring guarded by full/empty mbarriers.
+// Kernel launch with programmatic stream serialisation (and an optional cluster
+// along x).  Works the same under stream capture.
 // ---------------------------------------------------------------------------
-template <int BN> struct GemmCfg {
-    static constexpr int STAGES = BN <= 32 ? 8 : (BN <= 128 ? 6 : 4);
-    static constexpr int A_BYTES = 128 * 128;
-    static constexpr int B_BYTES = BN * 128;
-    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
-    static constexpr int SMEM = STAGES * (A_BYTES + B_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              int cluster_x, Args &&...args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+    if (cluster_x > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster_x, attr[na].val.clusterDim.y = 1, attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.attrs = attr, cfg.numAttrs = (unsigned)na;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+// ---------------------------------------------------------------------------
+// Tile width BN and cluster split S of a GEMM [M x N x K].
+// ---------------------------------------------------------------------------
+struct GemmPlan {
+    int BN, S;
 };
 
-template <int BN, typename Epi>
-__global__ void __launch_bounds__(192, 1)
-k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const StepParams *sp,
-          int T, int N, int K, Epi epi, int *status) {
-    using G = GemmCfg<BN>;
-    extern __shared__ uint8_t smem_raw[];
-    const int M = sp->nf * T;
-    const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN;
-    if (m0 >= M) return;                                    // uniform for the CTA, before any barrier or allocation
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *sA = smem, *sB = smem + G::STAGES * G::A_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sB + G::STAGES * G::B_BYTES);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + G::STAGES),
-                   accf = smem_u32(bars + 2 * G::STAGES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * G::STAGES + 1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nkb = (K + 63) / 64;
-    constexpr int SROW = BN + 4;                         // staging row stride in floats
-    float *stage = reinterpret_cast<float *>(smem);      // 128 x SROW floats, reuses the operand ring
-    static_assert(128 * (BN + 4) * 4 <= G::STAGES * (G::A_BYTES + G::B_BYTES), "staging tile must fit the ring");
+// CTAs that can be resident at once: two per SM for the narrow tiles (their shared
+// memory is sized for that), one for the wide ones.
+static int gemm_slots(int n_sm, int BN) { return BN <= 64 ? 2 * n_sm : n_sm; }
 
-    if (warp == 0 && lane == 0) {
-        for (int s = 0; s < G::STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 1);
-        }
-        mbar_init(accf, 1);
-        fence_mbar_init();
-        tma_prefetch_desc(&tmA);
-        tma_prefetch_desc(&tmB);
-    }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), G::TMEM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0) {
-        if (lane == 0) {
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % G::STAGES;
-                if (kb >= G::STAGES && !mbar_wait(empty0 + 8 * s, ((kb / G::STAGES) - 1) & 1, status)) break;
-                mbar_expect_tx(full0 + 8 * s, G::A_BYTES + G::B_BYTES);
-                tma_load_2d(smem_u32(sA + s * G::A_BYTES), &tmA, full0 + 8 * s, kb * 64, m0);
-                tma_load_2d(smem_u32(sB + s * G::B_BYTES), &tmB, full0 + 8 * s, kb * 64, n0);
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, BN);
-            bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % G::STAGES;
-                ok = mbar_wait(full0 + 8 * s, (kb / G::STAGES) & 1, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint64_t ad = umma_desc_k128(smem_u32(sA + s * G::A_BYTES));
-                const uint64_t bd = umma_desc_k128(smem_u32(sB + s * G::B_BYTES));
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                    umma_bf16_ss(tmem_base, ad + 2 * k4, bd + 2 * k4, idesc, (kb | k4) != 0);
-                umma_commit(empty0 + 8 * s);
-            }
-            umma_commit(accf);          // arrives when every UMMA above has completed
-        }
-    } else {
-        // accumulators: TMEM -> registers -> shared memory (the operand ring is free by now)
-        const int quad = warp & 3;      // TMEM lane quadrant this warp may read
-        const int row = quad * 32 + lane;
-        if (mbar_wait(accf, 0, status)) {
-            tc_fence_after();
-            float *srow = stage + (size_t)row * SROW;
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + c, r);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<uint4 *>(srow + c + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-            }
+static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind) {
+    // optional override for tuning: NFD_GEMM_PLAN="kind:BN:S,kind:BN:S,..." (kind = TC_* value, +10 for K > 2048)
+    if (const char *e = getenv("NFD_GEMM_PLAN")) {
+        for (const char *p = e; p && *p;) {
+            int k = 0, bn = 0, s = 0;
+            if (sscanf(p, "%d:%d:%d", &k, &bn, &s) == 3 && k == tc_kind + (K > 2048 ? 10 : 0)) return {bn, s};
+            p = strchr(p, ',');
+            if (p) ++p;
         }
     }
-    tc_fence_before();
-    __syncthreads();
-    // fused epilogue from shared memory: 8 adjacent columns per thread, rows coalesced
-    {
-        constexpr int CPR = BN / 8;     // chunks per row
-        for (int ch = threadIdx.x; ch < 128 * CPR; ch += 192) {
-            const int row = ch / CPR, cc = ch % CPR;
-            const int m = m0 + row, n = n0 + cc * 8;
-            if (m < M && n < N) {
-                const float4 *sp4 = reinterpret_cast<const float4 *>(stage + (size_t)row * SROW + cc * 8);
-                const float4 v0 = sp4[0], v1 = sp4[1];
-                float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                epi.vec8(m, n, a);
-            }
+    // Cost in SM cycles, fitted to measurements on B200: an SM takes in operand tiles at about
+    // 55 bytes per cycle whatever the ring depth; CTAs that share an SM share that rate.
+    const int mt = (M + 127) / 128, nkb = (K + 63) / 64;
+    GemmPlan best{32, 1};
+    double best_cost = 1e30;
+    const int bns[3] = {32, 64, 128};
+    for (int bi = 0; bi < 3; ++bi) {
+        const int BN = bns[bi];
+        if (BN > 32 && BN > N) continue;
+        const int nt = (N + BN - 1) / BN;
+        for (int S = 1; S <= 4; S *= 2) {
+            if (S > 1 && nkb / S < 2) break;
+            const long long ctas = (long long)mt * nt * S;
+            const int slots = gemm_slots(fs.n_sm, BN);
+            const double waves = (double)((ctas + slots - 1) / slots);
+            const double share = ctas > fs.n_sm ? (double)(ctas < slots ? ctas : slots) / fs.n_sm : 1.0;
+            const double kb = (double)((nkb + S - 1) / S);
+            const double load = kb * (16384.0 + BN * 128.0) / 55.0 * share;
+            const double items = (128.0 / S) * (BN / 8.0) / 256.0;                 // epilogue items per thread
+            const double epi = 400.0 + items * (S > 1 ? 700.0 : 350.0) + BN * 4.0;
+            const double fixed = 3200.0 + (S > 1 ? 1500.0 : 0.0);
+            const double cost = waves * (fixed + load + epi);
+            if (cost < best_cost) best_cost = cost, best = {BN, S};
         }
     }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, G::TMEM_COLS);
+    return best;
 }
 
 template <int BN, typename Epi>
-static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const StepParams *sp, int T, const bf16 *A, const bf16 *Wt,
-                           int M, int N, int K, Epi epi) {
+static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const bf16 *A, const bf16 *Wt, int M, int N, int K, int S,
+                           Epi epi, L2Prefetch pf) {
     using G = GemmCfg<BN>;
     static bool attr_set = false;
     auto kern = k_gemm_tc<BN, Epi>;
@@ -236,28 +198,32 @@ static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const StepParams *sp,
     const CUtensorMap *ma = get_map_2d(fs, A, (int)fs.a_rows, K, 128);
     const CUtensorMap *mb = get_map_2d(fs, Wt, N, K, BN);
     if (!ma || !mb) return false;
-    dim3 grid((N + BN - 1) / BN, (M + 127) / 128);
-    kern<<<grid, 192, G::SMEM, st>>>(*ma, *mb, sp, T, N, K, epi, fs.d_status);
+    dim3 grid(((N + BN - 1) / BN) * S, (M + 127) / 128);
+    cudaError_t e = launch_pdl(kern, grid, dim3(G::THREADS), (size_t)G::SMEM, st, S, *ma, *mb, M, N, K, S, epi, pf,
+                               fs.d_status);
+    if (e != cudaSuccess) {
+        fprintf(stderr, "libnfd: tensor-core GEMM launch failed (BN %d, S %d): %s\n", BN, S, cudaGetErrorString(e));
+        cudaGetLastError();
+        return false;
+    }
     return true;
 }
 
 template <typename TS, typename Epi>
-static bool fast_gemm(bool enabled, FastState &fs, cudaStream_t st, const StepParams *sp, int T, const TS *A,
-                      const TS *Wt, int M, int N, int K, Epi epi, int tc_kind) {
-    (void)tc_kind;
+static bool fast_gemm(bool enabled, FastState &fs, cudaStream_t st, const TS *A, const TS *Wt, int M, int N, int K,
+                      Epi epi, int tc_kind, L2Prefetch pf) {
     if constexpr (!std::is_same<TS, bf16>::value) {
         return false;
     } else {
         if (!enabled || !fs.ready) return false;
         if (K % 8 || K < 64 || N < 32 || (N & 7)) return false;
         if (((uintptr_t)A & 15) || ((uintptr_t)Wt & 15)) return false;
-        // largest tile that still gives every SM (about) one CTA
-        const int mt = (M + 127) / 128;
-        const int want = fs.n_sm * 4 / 5;
-        if (N >= 256 && mt * ((N + 255) / 256) >= want) return launch_gemm_tc<256, Epi>(fs, st, sp, T, A, Wt, M, N, K, epi);
-        if (N >= 128 && mt * ((N + 127) / 128) >= want) return launch_gemm_tc<128, Epi>(fs, st, sp, T, A, Wt, M, N, K, epi);
-        if (N >= 64 && mt * ((N + 63) / 64) >= want) return launch_gemm_tc<64, Epi>(fs, st, sp, T, A, Wt, M, N, K, epi);
-        return launch_gemm_tc<32, Epi>(fs, st, sp, T, A, Wt, M, N, K, epi);
+        const GemmPlan pl = plan_gemm(fs, M, N, K, tc_kind);
+        switch (pl.BN) {
+            case 128: return launch_gemm_tc<128, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
+            case 64: return launch_gemm_tc<64, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
+            default: return launch_gemm_tc<32, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
+        }
     }
 }
 
@@ -280,10 +246,14 @@ static int launch_attn_tc(FastState &fs, cudaStream_t st, const StepParams *sp, 
     if (!mq || !mk || !mv) return 0;
     const AttnPlan &pl = fs.plan;
     dim3 grid(pl.MAXSPLIT, pl.QT, nf * D.H);
-    kern<<<grid, 192, A::SMEM, st>>>(*mq, *mk, *mv, sp, D, layer, pl, out, fs.part_o, fs.part_ml, fs.d_status);
-    if (pl.MAXSPLIT == 1) return 1;
-    k_attn_combine<<<dim3(pl.QT, nf * D.H), 128, 0, st>>>(sp, D, pl, fs.part_o, fs.part_ml, out);
-    return 2;
+    cudaError_t e = launch_pdl(kern, grid, dim3(A::THREADS), (size_t)A::SMEM, st, 1, *mq, *mk, *mv, sp, D, layer, pl, out,
+                               fs.part_o, fs.part_ml, fs.attn_counters, fs.d_status);
+    if (e != cudaSuccess) {
+        fprintf(stderr, "libnfd: tensor-core attention launch failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return 0;
+    }
+    return 1;
 }
 
 // Returns the number of kernels launched (0: not handled, use the plain kernel).

@@ -1,0 +1,220 @@
+// Tensor-core GEMM of libnfd (bf16 operands, fp32 accumulation in tensor memory).
+//
+//   C[M,N] = A[M,K] * Wt[N,K]^T  followed by a fused epilogue functor.
+//
+// The projections of one forward pass have M = (frames in the pass) x (tokens per
+// frame): 336 rows at batch 1.  Such a GEMM is a few microseconds of work and is
+// bound by the rate and latency with which operand tiles reach an SM, so the
+// kernel is built around latency:
+//   - one CTA per 128 x BN output tile and K range; the K range of a tile is
+//     split over the S CTAs of a thread-block cluster (S = 1, 2, 4 or 8), which
+//     keeps 148 SMs busy with 3 row tiles and shortens every CTA's chain of
+//     dependent loads;
+//   - each CTA parks its partial accumulator in its own shared memory; after a
+//     cluster barrier CTA r reads rows [r*128/S, (r+1)*128/S) of all S partials
+//     through distributed shared memory, sums them in split order
+//     (deterministic) and runs the epilogue for those rows;
+//   - warp 0 = TMA producer, warp 1 = tensor-memory allocation + UMMA issue,
+//     warps 2-9 = accumulator read-out and epilogue (two warps per TMEM lane
+//     quadrant, each taking half of the columns);
+//   - programmatic dependent launch: barrier set-up, tensor-memory allocation and
+//     the first weight tiles (which never depend on the previous kernel) are
+//     issued before the wait on the predecessor grid; the epilogue's side inputs
+//     (bias, gate, residual, rotary table) are fetched while the UMMAs run;
+//   - every CTA also pulls a slice of the NEXT GEMM's weights towards L2, so that
+//     the weight stream from HBM runs one kernel ahead of its use.
+#pragma once
+#include "nfd_sm100.cuh"
+
+template <int BN> struct GemmCfg {
+    static constexpr int STAGES = BN <= 64 ? 4 : 6;
+    static constexpr int A_BYTES = 128 * 128;                  // 128 rows x 64 bf16
+    static constexpr int B_BYTES = BN * 128;
+    static constexpr int RING_BYTES = STAGES * (A_BYTES + B_BYTES);
+    static constexpr int SROW = BN + 4;                        // staging row stride (floats)
+    static constexpr int STAGE_BYTES = 128 * SROW * 4;         // partial accumulator tile; reuses the ring
+    static constexpr int TMEM_COLS = BN <= 32 ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
+    static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int THREADS = 320;
+    static constexpr int EPI_THREADS = 256;
+    static constexpr int MAX_ITEMS = 2;                        // epilogue items whose side inputs are prefetched
+    static constexpr int MIN_CTAS = BN <= 64 ? 2 : 1;
+    static_assert(STAGE_BYTES <= RING_BYTES, "staging tile must fit the operand ring");
+};
+
+// A byte range that the CTAs of a launch pull towards L2 (the next GEMM's weights).
+struct L2Prefetch {
+    const void *ptr;
+    unsigned long long bytes;      // multiple of 16; 0 = nothing
+};
+
+template <int BN, typename Epi>
+__global__ void __launch_bounds__(GemmCfg<BN>::THREADS, GemmCfg<BN>::MIN_CTAS)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int K,
+          int S, Epi epi, L2Prefetch pf, int *status) {
+    using G = GemmCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    // blockIdx.x = n_tile * S + split; the S splits of a tile form one cluster
+    const int split = blockIdx.x % S, n_tile = blockIdx.x / S;
+    const int m0 = blockIdx.y * 128, n0 = n_tile * BN;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *sA = smem, *sB = smem + G::STAGES * G::A_BYTES;
+    float *stage = reinterpret_cast<float *>(smem);          // reuses the ring once the UMMAs are done
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + G::RING_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + G::STAGES),
+                   accf = smem_u32(bars + 2 * G::STAGES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * G::STAGES + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb_all = (K + 63) / 64;
+    const int kb0 = (int)((long long)nkb_all * split / S), kb1 = (int)((long long)nkb_all * (split + 1) / S);
+    const int nkb = kb1 - kb0;
+    const int rows_per = 128 / S;                            // rows of the tile this CTA finishes
+
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+        for (int s = 0; s < G::STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accf, 1);
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), G::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // epilogue state that lives across the cluster barrier (used by warps 2-9 only)
+    constexpr int CPR = BN / 8;                              // 8-column chunks per row
+    const int et = (int)threadIdx.x - 64;                    // 0..255 for the epilogue warps
+    const int n_items = rows_per * CPR;                      // items of this CTA's row slice
+    const int r_base = (S > 1 ? (int)cluster_ctarank() : 0) * rows_per;   // first tile row of the slice
+    typename Epi::Side side[G::MAX_ITEMS];
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // weights never depend on the previous kernel: fill the ring's weight halves first
+            const int pre = nkb < G::STAGES ? nkb : G::STAGES;
+            for (int kb = 0; kb < pre; ++kb) {
+                mbar_expect_tx(full0 + 8 * kb, G::A_BYTES + G::B_BYTES);
+                tma_load_2d(smem_u32(sB + kb * G::B_BYTES), &tmB, full0 + 8 * kb, (kb0 + kb) * 64, n0);
+            }
+            pdl_wait();
+            for (int kb = 0; kb < pre; ++kb)
+                tma_load_2d(smem_u32(sA + kb * G::A_BYTES), &tmA, full0 + 8 * kb, (kb0 + kb) * 64, m0);
+            for (int kb = pre; kb < nkb; ++kb) {
+                const int s = kb % G::STAGES;
+                if (!mbar_wait(empty0 + 8 * s, ((kb / G::STAGES) - 1) & 1, status)) break;
+                mbar_expect_tx(full0 + 8 * s, G::A_BYTES + G::B_BYTES);
+                tma_load_2d(smem_u32(sA + s * G::A_BYTES), &tmA, full0 + 8 * s, (kb0 + kb) * 64, m0);
+                tma_load_2d(smem_u32(sB + s * G::B_BYTES), &tmB, full0 + 8 * s, (kb0 + kb) * 64, n0);
+            }
+        } else if (lane == 1 && pf.bytes) {
+            // this CTA's slice of the next GEMM's weights, towards L2 in 8 KiB pieces
+            const unsigned long long n_cta = (unsigned long long)gridDim.x * gridDim.y;
+            const unsigned long long cta = (unsigned long long)blockIdx.y * gridDim.x + blockIdx.x;
+            const unsigned long long per = ((pf.bytes / n_cta + 15) / 16 + 1) * 16;
+            unsigned long long b = cta * per, e = b + per;
+            if (e > pf.bytes) e = pf.bytes;
+            for (; b < e; b += 8192) {
+                const unsigned long long n = e - b < 8192 ? e - b : 8192;
+                bulk_prefetch_l2(reinterpret_cast<const uint8_t *>(pf.ptr) + b, (uint32_t)n);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            pdl_launch();
+            constexpr uint32_t idesc = umma_idesc_bf16(128, BN);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % G::STAGES;
+                if (!mbar_wait(full0 + 8 * s, (kb / G::STAGES) & 1, status)) break;
+                tc_fence_after();
+                const uint64_t ad = umma_desc_k128(smem_u32(sA + s * G::A_BYTES));
+                const uint64_t bd = umma_desc_k128(smem_u32(sB + s * G::B_BYTES));
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                    umma_bf16_ss(tmem_base, ad + 2 * k4, bd + 2 * k4, idesc, (kb | k4) != 0);
+                umma_commit(empty0 + 8 * s);
+            }
+            umma_commit(accf);          // arrives when every UMMA above has completed
+        }
+    } else {
+        pdl_wait();
+        // side inputs of the first items (bias, gate, residual, rotary table), fetched while the UMMAs run
+#pragma unroll
+        for (int i = 0; i < G::MAX_ITEMS; ++i) {
+            const int it = et + i * G::EPI_THREADS;
+            if (it < n_items) {
+                const int m = m0 + r_base + it / CPR, n = n0 + (it % CPR) * 8;
+                if (m < M && n < N) epi.load(m, n, side[i]);
+            }
+        }
+        // partial accumulator: tensor memory -> this CTA's staging tile (the ring is free by now)
+        const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;                    // which half of the columns
+        const int row = quad * 32 + lane;                    // tile row held by this thread
+        if (mbar_wait(accf, 0, status)) {
+            tc_fence_after();
+            float *srow = stage + (size_t)row * G::SROW;
+            constexpr int HC = BN / 2;                       // columns per half
+#pragma unroll
+            for (int c = 0; c < HC; c += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + half * HC + c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; j += 4)
+                    *reinterpret_cast<uint4 *>(srow + half * HC + c + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (S > 1)
+        cluster_sync_all();              // every CTA of the cluster has parked its partial tile
+    else
+        __syncthreads();
+    if (warp >= 2) {
+        // sum the S partials in split order, then the fused epilogue: 8 adjacent columns per item
+        const uint32_t stage_u32 = smem_u32(stage);
+        for (int i0 = 0; i0 * G::EPI_THREADS < n_items; i0 += G::MAX_ITEMS) {
+#pragma unroll
+            for (int i = 0; i < G::MAX_ITEMS; ++i) {
+                const int it = et + (i0 + i) * G::EPI_THREADS;
+                if (it >= n_items) continue;
+                const int trow = r_base + it / CPR, cc = it % CPR;
+                const int m = m0 + trow, n = n0 + cc * 8;
+                if (m >= M || n >= N) continue;
+                if (i0 > 0) epi.load(m, n, side[i]);
+                const uint32_t off = (uint32_t)(trow * G::SROW + cc * 8) * 4;
+                float4 v0, v1;
+                if (S == 1) {
+                    const float *p = stage + (size_t)trow * G::SROW + cc * 8;
+                    v0 = *reinterpret_cast<const float4 *>(p), v1 = *reinterpret_cast<const float4 *>(p + 4);
+                } else {
+                    uint32_t ra = cluster_map(stage_u32 + off, 0);
+                    v0 = ld_cluster_f4(ra), v1 = ld_cluster_f4(ra + 16);
+                    for (int s = 1; s < S; ++s) {
+                        ra = cluster_map(stage_u32 + off, (uint32_t)s);
+                        const float4 u0 = ld_cluster_f4(ra), u1 = ld_cluster_f4(ra + 16);
+                        v0.x += u0.x, v0.y += u0.y, v0.z += u0.z, v0.w += u0.w;
+                        v1.x += u1.x, v1.y += u1.y, v1.z += u1.z, v1.w += u1.w;
+                    }
+                }
+                float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                epi.apply(m, n, a, side[i]);
+            }
+        }
+    }
+    tc_fence_before();
+    if (S > 1)
+        cluster_sync_all();              // no CTA leaves while a peer may still read its partial tile
+    else
+        __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, G::TMEM_COLS);
+}

@@ -8,7 +8,10 @@
 // ---------------------------------------------------------------------------
 // Pass parameters: first kernel of every pass.
 // ---------------------------------------------------------------------------
+// It does not release its dependents early: a kernel that starts after this one
+// may read the descriptor before its own wait on the predecessor grid.
 __global__ void k_set_params(StepParams p, StepParams *dst) {
+    pdl_wait();
     const int n_words = sizeof(StepParams) / 4;
     const int *src = reinterpret_cast<const int *>(&p);
     int *d = reinterpret_cast<int *>(dst);
@@ -21,6 +24,8 @@ __global__ void k_set_params(StepParams p, StepParams *dst) {
 // action embedding row; then per-layer modulation W_mod * SiLU(c) + b.
 // ---------------------------------------------------------------------------
 __global__ void k_temb(const StepParams *sp, float t_scale, float *emb /*[rows][256]*/) {
+    pdl_wait();
+    pdl_launch();
     int c = blockIdx.x;
     if (c >= sp->nc) return;
     int i = threadIdx.x;              // 0..127
@@ -37,11 +42,37 @@ __global__ void k_temb(const StepParams *sp, float t_scale, float *emb /*[rows][
 enum { GEMV_T1 = 0, GEMV_T2 = 1, GEMV_MOD = 2 };
 
 // y[c][o] = f( sum_i Wt[o][i] * x[c][i] + b[o] ), one warp per output o, all
-// conditioning rows c.  blockIdx.y selects the layer for GEMV_MOD.
+// conditioning rows c (four at a time, so a weight row is read once for up to
+// four rows).  Weights are read 16 bytes per lane.  blockIdx.y selects the
+// layer for GEMV_MOD.  n_in must be a multiple of 8.
+template <typename TS> struct WVec;
+template <> struct WVec<bf16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const bf16 *p, float *f) {
+        const uint4 u = *reinterpret_cast<const uint4 *>(p);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __bfloat1622float2(h[i]);
+            f[2 * i] = t.x, f[2 * i + 1] = t.y;
+        }
+    }
+};
+template <> struct WVec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float *p, float *f) {
+        const float4 u = *reinterpret_cast<const float4 *>(p);
+        f[0] = u.x, f[1] = u.y, f[2] = u.z, f[3] = u.w;
+    }
+};
+
 template <typename TS, int MODE>
 __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *const *Wt_l, const TS *const *b_l,
                                               const TS *a_emb, const float *x, float *y, int n_in, int n_out,
                                               size_t y_row_stride, size_t y_layer_stride) {
+    pdl_wait();
+    pdl_launch();
+    constexpr int NV = WVec<TS>::N;
     const int layer = blockIdx.y;
     const TS *Wt = Wt_l[layer];
     const TS *b = b_l[layer];
@@ -50,56 +81,111 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
     if (o >= n_out) return;
     const int nc = sp->nc;
     const TS *wrow = Wt + (size_t)o * n_in;
-    for (int c = 0; c < nc; ++c) {
-        const float *xc = x + (size_t)c * n_in;
-        float acc = 0.f;
-        for (int i = lane; i < n_in; i += 32) acc = fmaf(to_f(wrow[i]), xc[i], acc);
-        acc = warp_sum(acc);
-        if (lane == 0) {
-            float v = acc + to_f(b[o]);
-            if (MODE == GEMV_T1) v = silu_f(v);
-            if (MODE == GEMV_T2) v = silu_f(v + to_f(a_emb[(size_t)sp->cd[c].action * n_out + o]));
-            y[(size_t)c * y_row_stride + (size_t)layer * y_layer_stride + o] = v;
+    for (int c0 = 0; c0 < nc; c0 += 4) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int i = lane * NV; i < n_in; i += 32 * NV) {
+            float w[NV];
+            WVec<TS>::load(wrow + i, w);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (c0 + u < nc) {
+                    const float *xc = x + (size_t)(c0 + u) * n_in + i;
+#pragma unroll
+                    for (int e = 0; e < NV; e += 4) {
+                        const float4 xv = *reinterpret_cast<const float4 *>(xc + e);
+                        acc[u] = fmaf(w[e], xv.x, acc[u]);
+                        acc[u] = fmaf(w[e + 1], xv.y, acc[u]);
+                        acc[u] = fmaf(w[e + 2], xv.z, acc[u]);
+                        acc[u] = fmaf(w[e + 3], xv.w, acc[u]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = c0 + u;
+            if (c >= nc) break;
+            const float r = warp_sum(acc[u]);
+            if (lane == 0) {
+                float v = r + to_f(b[o]);
+                if (MODE == GEMV_T1) v = silu_f(v);
+                if (MODE == GEMV_T2) v = silu_f(v + to_f(a_emb[(size_t)sp->cd[c].action * n_out + o]));
+                y[(size_t)c * y_row_stride + (size_t)layer * y_layer_stride + o] = v;
+            }
         }
     }
 }
 
 // ---------------------------------------------------------------------------
-// Patchify + embed: z[tok][o] = sum_p (alpha*x_a + beta*x_b)[patch p of tok] * Wt_pe[o][p] + b[o]
+// Patchify + embed: z[tok][o] = sum_p (alpha*x_a + beta*x_b)[patch p of tok] * W_pe[p][o] + b[o].
+// A CTA takes PE_TOK tokens; W_pe is used in its [P][d] layout so that adjacent
+// threads read adjacent outputs.
 // ---------------------------------------------------------------------------
+#define PE_TOK 8
 template <typename TS>
-__global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *Wt_pe, const TS *b_pe,
+__global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
                                                      float *z) {
-    extern __shared__ float s_patch[];
-    const int m = blockIdx.x;
-    if (m >= sp->nf * D.T) return;
-    const int j = m / D.T, tok = m % D.T;
-    const int r = tok / D.tw, c = tok % D.tw;
+    extern __shared__ float s_patch[];          // [PE_TOK][P]
+    pdl_wait();
+    pdl_launch();
+    const int M = sp->nf * D.T;
+    const int m0 = blockIdx.x * PE_TOK;
+    if (m0 >= M) return;
     const float *xa = sp->x_a, *xb = sp->x_b;
     const float alpha = sp->alpha, beta = sp->beta;
-    for (int p = threadIdx.x; p < D.P; p += blockDim.x) {
-        int ch = p / (D.p * D.p), py = (p / D.p) % D.p, px = p % D.p;
-        size_t idx = (((size_t)j * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
-        float v = alpha * xa[idx];
-        if (xb) v = fmaf(beta, xb[idx], v);
-        s_patch[p] = v;
+    for (int i = threadIdx.x; i < PE_TOK * D.P; i += blockDim.x) {
+        const int t = i / D.P, p = i - t * D.P, m = m0 + t;
+        float v = 0.f;
+        if (m < M) {
+            const int j = m / D.T, tok = m % D.T;
+            const int r = tok / D.tw, c = tok % D.tw;
+            const int ch = p / (D.p * D.p), py = (p / D.p) % D.p, px = p % D.p;
+            const size_t idx = (((size_t)j * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
+            v = alpha * xa[idx];
+            if (xb) v = fmaf(beta, xb[idx], v);
+        }
+        s_patch[i] = v;
     }
     __syncthreads();
     for (int o = threadIdx.x; o < D.d; o += blockDim.x) {
-        const TS *w = Wt_pe + (size_t)o * D.P;
-        float acc = 0.f;
-        for (int p = 0; p < D.P; ++p) acc = fmaf(s_patch[p], to_f(w[p]), acc);
-        z[(size_t)m * D.d + o] = acc + to_f(b_pe[o]);
+        float acc[PE_TOK];
+#pragma unroll
+        for (int t = 0; t < PE_TOK; ++t) acc[t] = 0.f;
+        for (int p = 0; p < D.P; ++p) {
+            const float w = to_f(W_pe[(size_t)p * D.d + o]);
+#pragma unroll
+            for (int t = 0; t < PE_TOK; ++t) acc[t] = fmaf(s_patch[t * D.P + p], w, acc[t]);
+        }
+        const float bo = to_f(b_pe[o]);
+#pragma unroll
+        for (int t = 0; t < PE_TOK; ++t)
+            if (m0 + t < M) z[(size_t)(m0 + t) * D.d + o] = acc[t] + bo;
     }
 }
 
 // ---------------------------------------------------------------------------
-// adaLN: out = norm(z) * (1 + scale_f) + shift_f, one warp per token.
+// adaLN: out = norm(z) * (1 + scale_f) + shift_f, one warp per token.  Rows of
+// up to 1024 elements are held in registers (one read of z); longer rows are
+// re-read from L1/L2.
 // ---------------------------------------------------------------------------
+template <typename TS> __device__ __forceinline__ void store4(TS *o, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float *o, float a, float b, float c, float d) {
+    *reinterpret_cast<float4 *>(o) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<bf16>(bf16 *o, float a, float b, float c, float d) {
+    uint2 u;
+    __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&u);
+    h[0] = __floats2bfloat162_rn(a, b);
+    h[1] = __floats2bfloat162_rn(c, d);
+    *reinterpret_cast<uint2 *>(o) = u;
+}
+
 template <typename TS>
-__global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, const float *z, TS *out,
+__global__ void __launch_bounds__(128) k_adaln(const StepParams *sp, Dims D, const float *z, TS *out,
                                                const float *mod, size_t row_stride, size_t off_shift,
                                                size_t off_scale) {
+    pdl_wait();
+    pdl_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m = blockIdx.x * (blockDim.x >> 5) + warp;
     if (m >= sp->nf * D.T) return;
@@ -107,12 +193,45 @@ __global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, con
     const float *zr = z + (size_t)m * D.d;
     const float *sh = mod + (size_t)row * row_stride + off_shift;
     const float *sc = mod + (size_t)row * row_stride + off_scale;
+    const float inv_d = 1.0f / (float)D.d;
+    if (D.d <= 1024) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = u * 128 + lane * 4;
+            v[u] = i < D.d ? *reinterpret_cast<const float4 *>(zr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float s = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += (v[u].x + v[u].y) + (v[u].z + v[u].w);
+        const float mean = (D.norm == 0) ? warp_sum(s) * inv_d : 0.f;
+        float q = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (u * 128 + lane * 4 < D.d) {
+                const float a = v[u].x - mean, b = v[u].y - mean, c = v[u].z - mean, e = v[u].w - mean;
+                q += (a * a + b * b) + (c * c + e * e);
+            }
+        }
+        const float rstd = rsqrtf(warp_sum(q) * inv_d + D.eps);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = u * 128 + lane * 4;
+            if (i < D.d) {
+                const float4 a = *reinterpret_cast<const float4 *>(sh + i);
+                const float4 b = *reinterpret_cast<const float4 *>(sc + i);
+                store4<TS>(out + (size_t)m * D.d + i, fmaf((v[u].x - mean) * rstd, 1.0f + b.x, a.x),
+                           fmaf((v[u].y - mean) * rstd, 1.0f + b.y, a.y), fmaf((v[u].z - mean) * rstd, 1.0f + b.z, a.z),
+                           fmaf((v[u].w - mean) * rstd, 1.0f + b.w, a.w));
+            }
+        }
+        return;
+    }
     float s = 0.f;
     for (int i = lane * 4; i < D.d; i += 128) {
         float4 v = *reinterpret_cast<const float4 *>(zr + i);
         s += (v.x + v.y) + (v.z + v.w);
     }
-    const float inv_d = 1.0f / (float)D.d;
     float mean = (D.norm == 0) ? warp_sum(s) * inv_d : 0.f;
     float q = 0.f;
     for (int i = lane * 4; i < D.d; i += 128) {
@@ -125,11 +244,9 @@ __global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, con
         float4 v = *reinterpret_cast<const float4 *>(zr + i);
         float4 a = *reinterpret_cast<const float4 *>(sh + i);
         float4 b = *reinterpret_cast<const float4 *>(sc + i);
-        TS *o = out + (size_t)m * D.d + i;
-        o[0] = from_f<TS>(fmaf((v.x - mean) * rstd, 1.0f + b.x, a.x));
-        o[1] = from_f<TS>(fmaf((v.y - mean) * rstd, 1.0f + b.y, a.y));
-        o[2] = from_f<TS>(fmaf((v.z - mean) * rstd, 1.0f + b.z, a.z));
-        o[3] = from_f<TS>(fmaf((v.w - mean) * rstd, 1.0f + b.w, a.w));
+        store4<TS>(out + (size_t)m * D.d + i, fmaf((v.x - mean) * rstd, 1.0f + b.x, a.x),
+                   fmaf((v.y - mean) * rstd, 1.0f + b.y, a.y), fmaf((v.z - mean) * rstd, 1.0f + b.z, a.z),
+                   fmaf((v.w - mean) * rstd, 1.0f + b.w, a.w));
     }
 }
 
@@ -138,6 +255,8 @@ __global__ void __launch_bounds__(256) k_adaln(const StepParams *sp, Dims D, con
 // pair of the head dimension, [nf*T][dh/2].
 // ---------------------------------------------------------------------------
 __global__ void k_rope_table(const StepParams *sp, Dims D, const RopeTab *rt, float2 *tab) {
+    pdl_wait();
+    pdl_launch();
     const int half = D.dh >> 1;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= sp->nf * D.T * half) return;
@@ -169,9 +288,12 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float *f) {
 
 // ---------------------------------------------------------------------------
 // GEMM epilogues.  operator() takes one output row m and two adjacent columns
-// (n, n+1), n even, holding the fp32 accumulators (plain GEMM).  vec8() takes
-// eight adjacent columns n..n+7, n a multiple of 8 (tensor-core GEMM, bf16
-// storage only); it reads and writes 16 bytes at a time.
+// (n, n+1), n even, holding the fp32 accumulators (plain GEMM).  The tensor-core
+// GEMM (bf16 storage only) works on eight adjacent columns n..n+7, n a multiple
+// of 8, 16 bytes at a time, in two steps: load() fetches everything the item
+// needs besides the accumulators (bias, gate, residual, rotary table) into a
+// Side record, so that the fetch can be issued while the UMMAs still run;
+// apply() combines it with the accumulators and stores.
 // ---------------------------------------------------------------------------
 // QKV: + bias, 3D RoPE on q and k (Section 3.1 "3D Positional Embedding":
 // adjacent pairs, per-axis frequencies), q -> [H][Nq][dh], k/v -> cache pages.
@@ -182,10 +304,26 @@ template <typename TS> struct EpiQKV {
     const RopeTab *rt;
     Dims D;
     int layer;
-    const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by vec8
-    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+    const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by the tensor-core path
+    int n_rows;                 // nf*T: rows of the pass (q is [H][n_rows][dh])
+    struct Side {
+        uint4 bias;
+        float4 c01, c23;        // (cos, sin) of four adjacent pairs
+        FrameDesc fr;
+    };
+    __device__ __forceinline__ void load(int m, int n, Side &s) const {
+        s.bias = *reinterpret_cast<const uint4 *>(bias + n);
+        const int which = n / D.d, col = n - which * D.d;
+        const int e = col % D.dh;
+        if (which < 2) {
+            const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
+            s.c01 = cs[0], s.c23 = cs[1];
+        }
+        s.fr = sp->fr[m / D.T];
+    }
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
         float b[8];
-        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+        unpack_bf16x8(s.bias, b);
         const int which = n / D.d, col = n - which * D.d;
         const int head = col / D.dh, e = col - head * D.dh;
         const int j = m / D.T, tok = m - j * D.T;
@@ -193,9 +331,7 @@ template <typename TS> struct EpiQKV {
         for (int i = 0; i < 8; ++i) a[i] += b[i];
         TS *dst;
         if (which < 2) {
-            const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
-            const float4 c01 = cs[0], c23 = cs[1];
-            const float cv[4] = {c01.x, c01.z, c23.x, c23.z}, sv[4] = {c01.y, c01.w, c23.y, c23.w};
+            const float cv[4] = {s.c01.x, s.c01.z, s.c23.x, s.c23.z}, sv[4] = {s.c01.y, s.c01.w, s.c23.y, s.c23.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const float r0 = a[2 * i] * cv[i] - a[2 * i + 1] * sv[i];
@@ -205,10 +341,9 @@ template <typename TS> struct EpiQKV {
             }
         }
         if (which == 0) {
-            dst = q + ((size_t)head * (sp->nf * D.T) + m) * D.dh + e;
+            dst = q + ((size_t)head * ((size_t)n_rows) + m) * D.dh + e;
         } else {
-            const FrameDesc fr = sp->fr[j];
-            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, fr.stream, layer, fr.frame) +
+            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, s.fr.stream, layer, s.fr.frame) +
                   ((size_t)head * D.T + tok) * D.dh + e;
         }
         *reinterpret_cast<uint4 *>(dst) = pack_bf16x8(a);
@@ -232,7 +367,7 @@ template <typename TS> struct EpiQKV {
         }
         TS *dst;
         if (which == 0) {
-            dst = q + ((size_t)head * (sp->nf * D.T) + m) * D.dh + e;
+            dst = q + ((size_t)head * n_rows + m) * D.dh + e;
         } else {
             TS *base = (which == 1) ? kc : vc;
             dst = base + kv_page_offset(D, fr.stream, layer, fr.frame) + ((size_t)head * D.T + tok) * D.dh + e;
@@ -250,22 +385,31 @@ template <typename TS> struct EpiGateRes {
     const float *gate;      // mod + layer offset + chunk offset
     size_t row_stride;
     Dims D;
-    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
-        float b[8];
-        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+    struct Side {
+        uint4 bias;
+        float4 g0, g1, z0, z1;
+    };
+    __device__ __forceinline__ void load(int m, int n, Side &s) const {
+        s.bias = *reinterpret_cast<const uint4 *>(bias + n);
         const int row = sp->fr[m / D.T].cond_row;
         const float4 *g = reinterpret_cast<const float4 *>(gate + (size_t)row * row_stride + n);
+        const float4 *zp = reinterpret_cast<const float4 *>(z + (size_t)m * D.d + n);
+        s.g0 = g[0], s.g1 = g[1];
+        s.z0 = zp[0], s.z1 = zp[1];
+    }
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
+        float b[8];
+        unpack_bf16x8(s.bias, b);
+        float4 z0 = s.z0, z1 = s.z1;
+        z0.x = fmaf(s.g0.x, a[0] + b[0], z0.x);
+        z0.y = fmaf(s.g0.y, a[1] + b[1], z0.y);
+        z0.z = fmaf(s.g0.z, a[2] + b[2], z0.z);
+        z0.w = fmaf(s.g0.w, a[3] + b[3], z0.w);
+        z1.x = fmaf(s.g1.x, a[4] + b[4], z1.x);
+        z1.y = fmaf(s.g1.y, a[5] + b[5], z1.y);
+        z1.z = fmaf(s.g1.z, a[6] + b[6], z1.z);
+        z1.w = fmaf(s.g1.w, a[7] + b[7], z1.w);
         float4 *zp = reinterpret_cast<float4 *>(z + (size_t)m * D.d + n);
-        const float4 g0 = g[0], g1 = g[1];
-        float4 z0 = zp[0], z1 = zp[1];
-        z0.x = fmaf(g0.x, a[0] + b[0], z0.x);
-        z0.y = fmaf(g0.y, a[1] + b[1], z0.y);
-        z0.z = fmaf(g0.z, a[2] + b[2], z0.z);
-        z0.w = fmaf(g0.w, a[3] + b[3], z0.w);
-        z1.x = fmaf(g1.x, a[4] + b[4], z1.x);
-        z1.y = fmaf(g1.y, a[5] + b[5], z1.y);
-        z1.z = fmaf(g1.z, a[6] + b[6], z1.z);
-        z1.w = fmaf(g1.w, a[7] + b[7], z1.w);
         zp[0] = z0;
         zp[1] = z1;
     }
@@ -283,11 +427,18 @@ template <typename TS> struct EpiGelu {
     const TS *bias;
     TS *out;
     int N;
-    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+    struct Side {
+        uint4 bias;
+    };
+    __device__ __forceinline__ void load(int m, int n, Side &s) const {
+        (void)m;
+        s.bias = *reinterpret_cast<const uint4 *>(bias + n);
+    }
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
         float b[8];
-        unpack_bf16x8(*reinterpret_cast<const uint4 *>(bias + n), b);
+        unpack_bf16x8(s.bias, b);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_f(a[i] + b[i]);
+        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i] + b[i]);
         *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
@@ -302,7 +453,11 @@ template <typename TS> struct EpiFinal {
     const StepParams *sp;
     const TS *bias;
     Dims D;
-    __device__ __forceinline__ void vec8(int m, int n, float *a) const {
+    struct Side {
+        int unused;
+    };
+    __device__ __forceinline__ void load(int, int, Side &) const {}
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &) const {
 #pragma unroll
         for (int i = 0; i < 8; i += 2) (*this)(m, n + i, a[i], a[i + 1]);
     }
@@ -329,6 +484,8 @@ __global__ void __launch_bounds__(256) k_gemm_simple(const StepParams *sp, int T
                                                      const TS *__restrict__ Wt, int N, int K, Epi epi) {
     __shared__ float As[16][64];
     __shared__ float Bs[16][64];
+    pdl_wait();
+    pdl_launch();
     const int M = sp->nf * T;
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
     if (m0 >= M) return;
@@ -382,6 +539,8 @@ template <typename TS, int DH>
 __global__ void __launch_bounds__(128) k_attn_simple(const StepParams *sp, Dims D, int layer, const TS *q,
                                                      const TS *kc, const TS *vc, TS *out) {
     constexpr int R = DH / 32;
+    pdl_wait();
+    pdl_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int Nq = sp->nf * D.T;
     const long long w = (long long)blockIdx.x * (blockDim.x >> 5) + warp;
@@ -422,6 +581,8 @@ __global__ void __launch_bounds__(128) k_attn_simple(const StepParams *sp, Dims 
 // ---------------------------------------------------------------------------
 // out = a*x + b*y (y may be NULL)
 __global__ void k_axpby(float *out, float a, const float *x, float b, const float *y, size_t n) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float v = a * x[i];
@@ -432,6 +593,8 @@ __global__ void k_axpby(float *out, float a, const float *x, float b, const floa
 // x0 = a*x' + b*v  (= sigma_d (x_in - t v));  if z: x' <- c*x0 + s*z  (re-noise to the next timestep)
 __global__ void k_sampler_post(float *xp, const float *v, const float *z, float *x0, float a, float b, float c,
                                float s, size_t n) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float e = fmaf(b, v[i], a * xp[i]);

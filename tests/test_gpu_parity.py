@@ -24,7 +24,12 @@ def dev(a):
     return torch.as_tensor(np.ascontiguousarray(a, dtype=np.float32)).cuda()
 
 
-def check(got, want, dtype, what=""):
+def check(got, want, dtype, what="", scale_by_magnitude=False):
+    """Max-abs and relative-L2 comparison.  scale_by_magnitude: the absolute bound is
+    multiplied by max(1, max|want|).  Used only for cached K/V pages of free-running
+    generation under the stress weights: those values reach |x| ~ 5, where one bf16
+    rounding step alone is 1.6e-2, and they are computed from frames the device
+    generated itself (each already within the latent tolerance)."""
     got = got.detach().float().cpu().numpy().astype(np.float64) if hasattr(got, "detach") else np.asarray(got, float)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape, (got.shape, want.shape)
@@ -32,6 +37,8 @@ def check(got, want, dtype, what=""):
     max_abs = np.abs(got - want).max()
     rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
     a, r = TOL[dtype]
+    if scale_by_magnitude:
+        a = a * max(1.0, float(np.abs(want).max()))
     assert max_abs <= a and rel <= r, f"{what}: max_abs={max_abs:.3e} (tol {a}), rel_l2={rel:.3e} (tol {r})"
     return max_abs, rel
 
@@ -140,8 +147,8 @@ def test_speculate_rollback_and_eviction(name, kind, opts):
     for l in range(cfg["n_layers"]):
         for f in range(orc.window_first(), orc.n_total):
             K, V = g.kv_read(l, f)
-            check(K, orc.kv_frame(l, f)[0], cfg["dtype"], f"K l{l} f{f}")
-            check(V, orc.kv_frame(l, f)[1], cfg["dtype"], f"V l{l} f{f}")
+            check(K, orc.kv_frame(l, f)[0], cfg["dtype"], f"K l{l} f{f}", scale_by_magnitude=True)
+            check(V, orc.kv_frame(l, f)[1], cfg["dtype"], f"V l{l} f{f}", scale_by_magnitude=True)
     assert g.status() == 0
 
 
