@@ -172,6 +172,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 const int g = b & 1, s = b % A::NST;
                 ok = mbar_wait(p_full + 8 * g, (b >> 1) & 1, status);
                 if (!ok) break;
+                // the group has consumed S(b): its next S goes first, so that it is ready as early as possible
+                if (b + 2 < nb) ok = issue_s(b + 2);
+                if (!ok) break;
                 tc_fence_after();
                 const uint64_t pd = umma_desc_k128(smem_u32(sP + g * A::P_BYTES));
                 const uint64_t vd = umma_desc_k128(smem_u32(sKV + s * 2 * A::KV_BYTES + A::KV_BYTES));
@@ -184,7 +187,6 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 }
                 umma_commit(pv_done + 8 * g);
                 umma_commit(kv_empty + 8 * s);
-                if (b + 2 < nb) ok = issue_s(b + 2);
             }
         }
     } else {
