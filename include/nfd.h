@@ -210,6 +210,13 @@ int nfd_status(nfd_ctx *ctx);
  * creation. */
 long long nfd_launch_count(nfd_ctx *ctx);
 
+/* The adaLN modulation of a frame (Section 3.1, "Action Conditioning") depends on
+ * its (FM time, action) pair only.  The library keeps the modulation of the most
+ * recently used pairs (96 of them) and computes a pair's modulation only when it
+ * is not there.  Returns how many pairs were found (hits) and how many had to be
+ * computed (misses) since creation; either pointer may be NULL. */
+int nfd_cond_cache_stats(nfd_ctx *ctx, long long *hits, long long *misses);
+
 /* Per-kernel timing.  Between nfd_profile_begin and nfd_profile_end every
  * kernel is launched directly (no graph replay) with a CUDA event before and
  * after it on the context's stream.  nfd_profile_end synchronises and returns,

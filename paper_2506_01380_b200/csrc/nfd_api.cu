@@ -68,6 +68,15 @@ struct nfd_ctx {
     FastState fs;
 
     std::vector<int> n_committed, n_tentative;
+    // Modulation cache: the adaLN modulation depends on (FM time, action) only, so each pair is computed
+    // once and kept in one of n_slots rows of `mod` / `fmod`; least recently used rows are replaced.
+    struct CondSlot {
+        unsigned t_bits = 0;
+        int action = -1;
+        long long last_use = -1;
+    };
+    std::vector<CondSlot> cond_slots;
+    long long pass_no = 0, cond_hits = 0, cond_misses = 0;
     std::map<int, GraphEntry> graphs;
 
     // per-kernel-class timing (nfd_profile_begin / nfd_profile_end)
@@ -158,7 +167,7 @@ static int validate_cfg(const nfd_cfg &g) {
     if (g.latent_c < 1 || g.latent_h < 1 || g.latent_w < 1 || g.patch < 1) return NFD_E_BADCFG;
     if (g.latent_h % g.patch || g.latent_w % g.patch) return NFD_E_BADCFG;
     int P = g.latent_c * g.patch * g.patch;
-    if (P % 2 || P > 1024) return NFD_E_BADCFG;
+    if (P % 2 || P > 512) return NFD_E_BADCFG;
     if ((size_t)g.latent_c * g.latent_h * g.latent_w % 4) return NFD_E_BADCFG;
     if (g.n_actions < 1 || g.ctx_frames < 0 || g.ctx_frames > 4096) return NFD_E_BADCFG;
     if (g.max_spec < 1 || g.max_spec > 8) return NFD_E_BADCFG;
@@ -179,6 +188,8 @@ static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
 // ---------------------------------------------------------------------------
 // One forward pass, enqueued on the context's stream.
 // ---------------------------------------------------------------------------
+#define NFD_COND_SLOTS 96       // rows of the modulation cache (> NFD_MAX_PASS_FRAMES)
+
 enum { CLS_PARAMS = 0, CLS_COND, CLS_PATCH, CLS_ADALN, CLS_GEMM_QKV, CLS_ATTN, CLS_GEMM_O, CLS_GEMM_FC1,
        CLS_GEMM_FC2, CLS_HEAD, CLS_SAMPLER, CLS_CACHE, CLS_COUNT };
 static const char *const kClassNames[CLS_COUNT] = {"params", "conditioning", "patch_embed", "adaln_norm",
@@ -270,27 +281,28 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     const int d = D.d, L = D.L, M = nf * D.T;
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
-    // conditioning
+    // conditioning: only for the (t, action) pairs that are not in the modulation cache
     c->cls = CLS_COND;
-    PLAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
-    PLAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
-            (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, (const float *)c->emb, c->h1, 256, d, (size_t)d,
-            (size_t)0);
-    PLAUNCH(c, (k_gemv<TS, GEMV_T2>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t2,
-            (const TS *const *)(c->dp_t2 + 1), (const TS *)c->a_emb, (const float *)c->h1, c->sc, d, d, (size_t)d,
-            (size_t)0);
-    PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((6 * d + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wmod,
-            (const TS *const *)c->dp_bmod, (const TS *)nullptr, (const float *)c->sc, c->mod, d, 6 * d, mod_row,
-            (size_t)6 * d);
-    if (kind == 0)
+    if (c->h_sp.nc > 0) {
+        PLAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
+        PLAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
+                (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, (const float *)c->emb, c->h1, 256, d, (size_t)d,
+                (size_t)0);
+        PLAUNCH(c, (k_gemv<TS, GEMV_T2>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t2,
+                (const TS *const *)(c->dp_t2 + 1), (const TS *)c->a_emb, (const float *)c->h1, c->sc, d, d, (size_t)d,
+                (size_t)0);
+        PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((6 * d + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wmod,
+                (const TS *const *)c->dp_bmod, (const TS *)nullptr, (const float *)c->sc, c->mod, d, 6 * d, mod_row,
+                (size_t)6 * d);
         PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((2 * d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_fmod,
                 (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, (const float *)c->sc, c->fmod, d, 2 * d,
                 (size_t)2 * d, (size_t)0);
+    }
     // tokens
     c->cls = CLS_PATCH;
     if (c->bf16_mode && c->fast)
         PLAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, (const RopeTab *)c->d_rope, c->rope_cs);
-    PLAUNCH(c, (k_patch_embed<TS>), (M + PE_TOK - 1) / PE_TOK, 256, PE_TOK * D.P * sizeof(float), sp, D,
+    PLAUNCH(c, (k_patch_embed<TS>), dim3((M + PE_TOK - 1) / PE_TOK, (d + 255) / 256), 256, PE_TOK * D.P * sizeof(float), sp, D,
             (const TS *)c->w_pe_io, (const TS *)c->b_pe, c->z);
     const int ln_grid = (M + 3) / 4;
     for (int l = 0; l < L; ++l) {
@@ -337,8 +349,18 @@ static void enqueue_body_any(nfd_ctx *c, int nf, int kind) {
         enqueue_body<float>(c, nf, kind);
 }
 
-// Run the pass described by c->h_sp.
+static int run_pass_inner(nfd_ctx *c);
+
+// Run the pass described by c->h_sp.  If it cannot be enqueued, the cache slots that it was to fill are
+// given up again.
 static int run_pass(nfd_ctx *c) {
+    const int rc = run_pass_inner(c);
+    if (rc != NFD_OK)
+        for (int r = 0; r < c->h_sp.nc; ++r) c->cond_slots[c->h_sp.cd[r].slot] = nfd_ctx::CondSlot();
+    return rc;
+}
+
+static int run_pass_inner(nfd_ctx *c) {
     const int nf = c->h_sp.nf, kind = c->h_sp.kind;
     if (!c->use_graph || c->st == nullptr || c->prof) {
         c->cls = CLS_PARAMS;
@@ -348,7 +370,7 @@ static int run_pass(nfd_ctx *c) {
         CK(c->launch_err);
         return NFD_OK;
     }
-    const int key = kind * 64 + nf + (c->fast ? 0 : 4096);
+    const int key = kind * 64 + nf + (c->fast ? 0 : 4096) + (c->h_sp.nc > 0 ? 0 : 8192);   // no conditioning kernels when all pairs are cached
     auto it = c->graphs.find(key);
     if (it == c->graphs.end()) {
         GraphEntry ge;
@@ -406,8 +428,17 @@ static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, 
         for (int j = 0; j < i; ++j)
             if (streams[j] == streams[i]) return NFD_E_RANGE;
     }
+    // validate everything before the modulation cache is touched: a failed call changes nothing
+    for (int i = 0; i < n; ++i) {
+        if (!(t[i] >= 0.f) || !(t[i] <= 1.f)) return NFD_E_RANGE;
+        for (int j = 0; j < (per_frame_actions ? k : 1); ++j) {
+            const int a = per_frame_actions ? actions[i * k + j] : actions[i];
+            if (a < 0 || a >= g.n_actions) return NFD_E_RANGE;
+        }
+    }
     StepParams &p = c->h_sp;
     memset(&p, 0, sizeof(p));
+    ++c->pass_no;
     p.nf = n * k;
     p.kind = kind;
     p.x_a = x_a, p.x_b = x_b, p.alpha = alpha, p.beta = beta, p.v_out = v_out;
@@ -415,16 +446,26 @@ static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, 
     for (int i = 0; i < n; ++i) {
         for (int j = 0; j < k; ++j) {
             int a = per_frame_actions ? actions[i * k + j] : actions[i];
-            if (a < 0 || a >= g.n_actions) return NFD_E_RANGE;
-            if (!(t[i] >= 0.f) || !(t[i] <= 1.f)) return NFD_E_RANGE;
-            int row = -1;
-            for (int r = 0; r < nc; ++r)
-                if (p.cd[r].action == a && p.cd[r].t == t[i]) row = r;
-            if (row < 0) {
-                row = nc++;
-                p.cd[row].t = t[i];
-                p.cd[row].action = a;
+            // modulation cache: reuse the slot of this (t, action) pair, else take the least recently used one
+            unsigned tb;
+            memcpy(&tb, &t[i], 4);
+            int row = -1, lru = -1;
+            for (int r = 0; r < (int)c->cond_slots.size(); ++r) {
+                const nfd_ctx::CondSlot &cs = c->cond_slots[r];
+                if (cs.action == a && cs.t_bits == tb) row = r;
+                if (cs.last_use != c->pass_no && (lru < 0 || cs.last_use < c->cond_slots[lru].last_use)) lru = r;
             }
+            if (row < 0) {
+                if (lru < 0 || nc >= NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;      // cannot happen: slots > frames per pass
+                row = lru;
+                c->cond_slots[row].t_bits = tb, c->cond_slots[row].action = a;
+                p.cd[nc].t = t[i], p.cd[nc].action = a, p.cd[nc].slot = row;
+                ++nc;
+                ++c->cond_misses;
+            } else if (c->cond_slots[row].last_use != c->pass_no) {
+                ++c->cond_hits;
+            }
+            c->cond_slots[row].last_use = c->pass_no;
             FrameDesc &f = p.fr[i * k + j];
             f.stream = streams[i];
             f.frame = c->n_total(streams[i]) + offset + j;
@@ -509,8 +550,10 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     A((void **)&c->emb, (size_t)NF * 256 * 4);
     A((void **)&c->h1, (size_t)NF * D.d * 4);
     A((void **)&c->sc, (size_t)NF * D.d * 4);
-    A((void **)&c->mod, (size_t)NF * D.L * 6 * D.d * 4);
-    A((void **)&c->fmod, (size_t)NF * 2 * D.d * 4);
+    const int n_slots = NFD_COND_SLOTS;
+    c->cond_slots.assign(n_slots, nfd_ctx::CondSlot());
+    A((void **)&c->mod, (size_t)n_slots * D.L * 6 * D.d * 4);
+    A((void **)&c->fmod, (size_t)n_slots * 2 * D.d * 4);
     A((void **)&c->xp, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->vbuf, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->d_sp, sizeof(StepParams));
@@ -783,6 +826,13 @@ int nfd_status(nfd_ctx *c) {
 }
 
 long long nfd_launch_count(nfd_ctx *c) { return c ? c->launches : 0; }
+
+int nfd_cond_cache_stats(nfd_ctx *c, long long *hits, long long *misses) {
+    if (!c) return NFD_E_NULLPTR;
+    if (hits) *hits = c->cond_hits;
+    if (misses) *misses = c->cond_misses;
+    return NFD_OK;
+}
 
 int nfd_profile_begin(nfd_ctx *c) {
     if (!c) return NFD_E_NULLPTR;

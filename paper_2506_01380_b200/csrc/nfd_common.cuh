@@ -12,14 +12,16 @@ struct FrameDesc {
     int stream;      // batch slot
     int frame;       // absolute frame index (RoPE position, ring slot = frame % R)
     int win_first;   // first frame this one attends to (>= 0, >= frame - W)
-    int cond_row;    // row of the conditioning / modulation tables
+    int cond_row;    // slot of the modulation cache that holds this frame's adaLN modulation
     int first_new;   // first frame of this stream whose K/V the current pass writes (earlier pages are final)
 };
 
-// One distinct (FM time, action) pair of a pass.
+// One (FM time, action) pair whose modulation this pass has to compute: the pairs
+// of a pass that are not in the modulation cache yet.
 struct CondDesc {
     float t;
     int action;
+    int slot;        // cache slot the result goes to
 };
 
 // Everything that changes from pass to pass.  Written to device memory by the
@@ -27,7 +29,7 @@ struct CondDesc {
 // values (cache position, timestep, action, I/O pointers).
 struct StepParams {
     int nf;                 // frames in this pass (tokens = nf * T)
-    int nc;                 // distinct conditioning rows
+    int nc;                 // conditioning rows to compute in this pass (0: every pair is cached)
     int kind;               // 0 denoise (all layers + velocity head), 1 commit (K/V only)
     int layer_for_attn;     // nfd_attention: which layer's pages hold the data
     const float *x_a;       // model input = alpha * x_a + beta * x_b

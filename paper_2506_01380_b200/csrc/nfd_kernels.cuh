@@ -110,7 +110,8 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
                 float v = r + to_f(b[o]);
                 if (MODE == GEMV_T1) v = silu_f(v);
                 if (MODE == GEMV_T2) v = silu_f(v + to_f(a_emb[(size_t)sp->cd[c].action * n_out + o]));
-                y[(size_t)c * y_row_stride + (size_t)layer * y_layer_stride + o] = v;
+                const int out_row = MODE == GEMV_MOD ? sp->cd[c].slot : c;     // modulation goes to its cache slot
+                y[(size_t)out_row * y_row_stride + (size_t)layer * y_layer_stride + o] = v;
             }
         }
     }
@@ -118,10 +119,13 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
 
 // ---------------------------------------------------------------------------
 // Patchify + embed: z[tok][o] = sum_p (alpha*x_a + beta*x_b)[patch p of tok] * W_pe[p][o] + b[o].
-// A CTA takes PE_TOK tokens; W_pe is used in its [P][d] layout so that adjacent
-// threads read adjacent outputs.
+// A CTA takes PE_TOK tokens (blockIdx.x) and 256 output columns (blockIdx.y).
+// Each thread owns one output column: it loads 64 rows of its W_pe column at a
+// time into registers (independent loads, all in flight together) and reuses
+// them for all tokens of the CTA.  W_pe is used in its [P][d] layout so that
+// adjacent threads read adjacent columns.
 // ---------------------------------------------------------------------------
-#define PE_TOK 8
+#define PE_TOK 16
 template <typename TS>
 __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
                                                      float *z) {
@@ -147,20 +151,40 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
         s_patch[i] = v;
     }
     __syncthreads();
-    for (int o = threadIdx.x; o < D.d; o += blockDim.x) {
-        float acc[PE_TOK];
+    const int o = blockIdx.y * blockDim.x + threadIdx.x;
+    if (o >= D.d) return;
+    float acc[PE_TOK];
 #pragma unroll
-        for (int t = 0; t < PE_TOK; ++t) acc[t] = 0.f;
+    for (int t = 0; t < PE_TOK; ++t) acc[t] = 0.f;
+    if (D.P % 64 == 0) {
+        for (int p0 = 0; p0 < D.P; p0 += 64) {
+            TS wr[64];
+#pragma unroll
+            for (int u = 0; u < 64; ++u) wr[u] = W_pe[(size_t)(p0 + u) * D.d + o];      // 64 independent loads
+#pragma unroll
+            for (int t = 0; t < PE_TOK; ++t) {
+                const float4 *sp_t = reinterpret_cast<const float4 *>(s_patch + t * D.P + p0);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const float4 x = sp_t[u];
+                    acc[t] = fmaf(x.x, to_f(wr[4 * u]), acc[t]);
+                    acc[t] = fmaf(x.y, to_f(wr[4 * u + 1]), acc[t]);
+                    acc[t] = fmaf(x.z, to_f(wr[4 * u + 2]), acc[t]);
+                    acc[t] = fmaf(x.w, to_f(wr[4 * u + 3]), acc[t]);
+                }
+            }
+        }
+    } else {
         for (int p = 0; p < D.P; ++p) {
             const float w = to_f(W_pe[(size_t)p * D.d + o]);
 #pragma unroll
             for (int t = 0; t < PE_TOK; ++t) acc[t] = fmaf(s_patch[t * D.P + p], w, acc[t]);
         }
-        const float bo = to_f(b_pe[o]);
-#pragma unroll
-        for (int t = 0; t < PE_TOK; ++t)
-            if (m0 + t < M) z[(size_t)(m0 + t) * D.d + o] = acc[t] + bo;
     }
+    const float bo = to_f(b_pe[o]);
+#pragma unroll
+    for (int t = 0; t < PE_TOK; ++t)
+        if (m0 + t < M) z[(size_t)(m0 + t) * D.d + o] = acc[t] + bo;
 }
 
 // ---------------------------------------------------------------------------

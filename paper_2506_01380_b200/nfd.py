@@ -43,7 +43,7 @@ EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_de
            "nfd_denoise_step_batched", "nfd_commit_frame", "nfd_speculate", "nfd_speculate_batched",
            "nfd_rollback", "nfd_kv_state", "nfd_kv_hash", "nfd_kv_read", "nfd_attention", "nfd_status",
            "nfd_launch_count", "nfd_set_option", "nfd_strerror", "nfd_profile_begin", "nfd_profile_end",
-           "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc"]
+           "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc", "nfd_cond_cache_stats"]
 
 
 class NfdError(RuntimeError):
@@ -89,6 +89,7 @@ def load():
     lib.nfd_profile_class_name.restype = C.c_char_p
     lib.nfd_attention_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                           vp, vp]
+    lib.nfd_cond_cache_stats.argtypes = [vp, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]
     lib.nfd_strerror.argtypes = [C.c_int]
     lib.nfd_strerror.restype = C.c_char_p
     _lib = lib
@@ -304,6 +305,12 @@ class NFD:
 
     def launch_count(self) -> int:
         return self.lib.nfd_launch_count(self._h)
+
+    def cond_cache_stats(self):
+        """(hits, misses) of the modulation cache since creation."""
+        h, m = C.c_longlong(), C.c_longlong()
+        _check(self.lib.nfd_cond_cache_stats(self._h, C.byref(h), C.byref(m)), "nfd_cond_cache_stats")
+        return int(h.value), int(m.value)
 
     def profile_begin(self):
         _check(self.lib.nfd_profile_begin(self._h), "nfd_profile_begin")

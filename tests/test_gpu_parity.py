@@ -274,3 +274,35 @@ def test_310m_slice_two_layers(kind):
 def test_310m_full_config_teacher_forced():
     """Config 3's shape: 24 layers, 16 context frames, one denoising pass, GPU vs oracle."""
     _teacher_forced(I.make_cfg("nfd310m"), "paper", n_prompt=16, k=1, seed=0)
+
+
+def test_modulation_cache_hits_evictions_and_values():
+    """The adaLN modulation is kept per (FM time, action) pair: a pass that finds its pair cached must
+    give bitwise the same velocity as a context that computes it afresh, also after the pair's slot was
+    replaced (more distinct pairs than slots) and recomputed."""
+    from paper_2506_01380_b200.nfd import NFD
+    torch = _torch()
+    cfg = I.make_cfg("tiny_bf16")
+    w = I.make_weights(cfg, 5, "stress")
+    g, orc = NFD(cfg, w), O.NFDOracle(cfg, w)
+    prompt(cfg, g, orc, 2, seed=900)
+    x = dev(I.round_bf16(I.make_latents(cfg, 1, 901)))
+    h0, m0 = g.cond_cache_stats()
+    v_first = g.denoise_step(x, 0.625, 3).clone()
+    assert g.cond_cache_stats() == (h0, m0 + 1)
+    v_again = g.denoise_step(x, 0.625, 3).clone()
+    assert g.cond_cache_stats() == (h0 + 1, m0 + 1)
+    assert torch.equal(v_first, v_again)
+    check(v_first, orc.denoise_step(x.cpu().numpy().astype(np.float64), 0.625, 3), cfg["dtype"], "velocity")
+    # more distinct pairs than the cache has slots: the first pair is replaced ...
+    for i in range(120):
+        g.denoise_step(x, float(np.float32(0.001 * (i + 1))), i % cfg["n_actions"])
+    h1, m1 = g.cond_cache_stats()
+    v_refill = g.denoise_step(x, 0.625, 3).clone()
+    assert g.cond_cache_stats() == (h1, m1 + 1), "the pair should have been evicted and recomputed"
+    assert torch.equal(v_first, v_refill)
+    # ... and a failed call leaves the cache as it was
+    with pytest.raises(Exception):
+        g.denoise_step(x, 0.3333, 99)
+    assert g.cond_cache_stats() == (h1, m1 + 1)
+    assert g.status() == 0
