@@ -876,6 +876,23 @@ int nfd_set_option(nfd_ctx *c, const char *name, int value) {
 }
 
 
+#ifdef NFD_TRACE
+// Timeline instrumentation (only in builds with -DNFD_TRACE): copy out the records gathered so far
+// (host buffer of `cap` records of 24 bytes: t0, t1, kind, sm), reset the buffer, return their number.
+int nfd_trace_read(nfd_ctx *c, void *host_buf, int cap) {
+    if (!c || !host_buf) return NFD_E_NULLPTR;
+    CK(cudaStreamSynchronize(c->st));
+    unsigned int n = 0;
+    CK(cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n)));
+    if (n > NFD_TRACE_CAP) n = NFD_TRACE_CAP;
+    if ((int)n > cap) n = (unsigned int)cap;
+    CK(cudaMemcpyFromSymbol(host_buf, g_trace, (size_t)n * sizeof(NfdTraceRec)));
+    const unsigned int zero = 0;
+    CK(cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero)));
+    return (int)n;
+}
+#endif
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------

@@ -72,6 +72,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
           float *part_o, float2 *part_ml, unsigned int *counters, int *status) {
     using A = AttnCfg<KB>;
     extern __shared__ uint8_t smem_raw[];
+    NFD_TRACE_T0();
     const int z = blockIdx.z, j = z / D.H, h = z % D.H;
     const int qt = blockIdx.y, split = blockIdx.x;
     // the pass descriptor was written by the first kernel of the pass, which completed long ago
@@ -405,4 +406,5 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, A::TMEM_COLS);
+    NFD_TRACE_END(TRK_ATTN);
 }

@@ -68,6 +68,53 @@ struct RopeTab {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- timeline instrumentation (compiled out unless NFD_TRACE is defined) ------
+// With -DNFD_TRACE every CTA of the instrumented kernels appends one record
+// (kernel kind, SM, start and end on the global nanosecond timer) to a buffer
+// that nfd_trace_read() copies out; the default build contains none of it.
+#ifdef NFD_TRACE
+#define NFD_TRACE_CAP (1 << 20)
+struct NfdTraceRec {
+    unsigned long long t0, t1;
+    int kind, sm;
+};
+__device__ NfdTraceRec g_trace[NFD_TRACE_CAP];
+__device__ unsigned int g_trace_n;
+__device__ __forceinline__ unsigned long long nfd_trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void nfd_trace_put(int kind, unsigned long long t0) {
+    const unsigned int i = atomicAdd(&g_trace_n, 1u);
+    if (i < NFD_TRACE_CAP) {
+        unsigned int sm;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+        g_trace[i].t0 = t0, g_trace[i].t1 = nfd_trace_now(), g_trace[i].kind = kind, g_trace[i].sm = (int)sm;
+    }
+}
+#define NFD_TRACE_T0() const unsigned long long nfd_t0_ = nfd_trace_now()
+#define NFD_TRACE_END(kind)                          \
+    do {                                             \
+        if (threadIdx.x == 0) nfd_trace_put((kind), nfd_t0_); \
+    } while (0)
+// a point event (t0 == t1 is the time of the call), e.g. right after the wait on the predecessor grid
+#define NFD_TRACE_MARK(kind)                                  \
+    do {                                                      \
+        if (threadIdx.x == 0) nfd_trace_put((kind), nfd_trace_now()); \
+    } while (0)
+#define NFD_TRACE_MARK_T(kind, tid)                           \
+    do {                                                      \
+        if (threadIdx.x == (tid)) nfd_trace_put((kind), nfd_trace_now()); \
+    } while (0)
+#else
+#define NFD_TRACE_T0() do { } while (0)
+#define NFD_TRACE_END(kind) do { } while (0)
+#define NFD_TRACE_MARK(kind) do { } while (0)
+#define NFD_TRACE_MARK_T(kind, tid) do { } while (0)
+#endif
+enum { TRK_PARAMS = 0, TRK_GEMV, TRK_PATCH, TRK_ADALN, TRK_GEMM, TRK_ATTN, TRK_OTHER };
+
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }

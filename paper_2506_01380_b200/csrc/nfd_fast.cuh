@@ -159,28 +159,41 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
     }
     // Cost in SM cycles, fitted to measurements on B200: an SM takes in operand tiles at about
     // 55 bytes per cycle whatever the ring depth; CTAs that share an SM share that rate.
-    const int mt = (M + 127) / 128, nkb = (K + 63) / 64;
-    GemmPlan best{32, 1};
-    double best_cost = 1e30;
+    // The split S is chosen for a one-frame pass (M = tokens per frame) and then kept for every M:
+    // the order in which the K range is summed, and with it every bit of the result, must not
+    // depend on how many frames share a pass.  Only the tile width follows M.
+    const int nkb = (K + 63) / 64;
+    auto cost_of = [&](int m_rows, int BN, int S) {
+        const int mt = (m_rows + 127) / 128, nt = (N + BN - 1) / BN;
+        const long long ctas = (long long)mt * nt * S;
+        const int slots = gemm_slots(fs.n_sm, BN);
+        const double waves = (double)((ctas + slots - 1) / slots);
+        const double share = ctas > fs.n_sm ? (double)(ctas < slots ? ctas : slots) / fs.n_sm : 1.0;
+        const double kb = (double)((nkb + S - 1) / S);
+        const double load = kb * (16384.0 + BN * 128.0) / 55.0 * share;
+        const double items = (128.0 / S) * (BN / 8.0) / 256.0;                 // epilogue items per thread
+        const double epi = 400.0 + items * (S > 1 ? 700.0 : 350.0) + BN * 4.0;
+        const double fixed = 3200.0 + (S > 1 ? 1500.0 : 0.0);
+        return waves * (fixed + load + epi);
+    };
     const int bns[3] = {32, 64, 128};
+    const int T = (int)(fs.a_rows / NFD_MAX_PASS_FRAMES);
+    int S_best = 1;
+    double best_cost = 1e30;
     for (int bi = 0; bi < 3; ++bi) {
-        const int BN = bns[bi];
-        if (BN > 32 && BN > N) continue;
-        const int nt = (N + BN - 1) / BN;
-        for (int S = 1; S <= 4; S *= 2) {
+        if (bns[bi] > 32 && bns[bi] > N) continue;
+        for (int S = 1; S <= GemmCfg<64>::MAX_S; S *= 2) {
             if (S > 1 && nkb / S < 2) break;
-            const long long ctas = (long long)mt * nt * S;
-            const int slots = gemm_slots(fs.n_sm, BN);
-            const double waves = (double)((ctas + slots - 1) / slots);
-            const double share = ctas > fs.n_sm ? (double)(ctas < slots ? ctas : slots) / fs.n_sm : 1.0;
-            const double kb = (double)((nkb + S - 1) / S);
-            const double load = kb * (16384.0 + BN * 128.0) / 55.0 * share;
-            const double items = (128.0 / S) * (BN / 8.0) / 256.0;                 // epilogue items per thread
-            const double epi = 400.0 + items * (S > 1 ? 700.0 : 350.0) + BN * 4.0;
-            const double fixed = 3200.0 + (S > 1 ? 1500.0 : 0.0);
-            const double cost = waves * (fixed + load + epi);
-            if (cost < best_cost) best_cost = cost, best = {BN, S};
+            const double c = cost_of(T, bns[bi], S);
+            if (c < best_cost) best_cost = c, S_best = S;
         }
+    }
+    GemmPlan best{32, S_best};
+    best_cost = 1e30;
+    for (int bi = 0; bi < 3; ++bi) {
+        if (bns[bi] > 32 && bns[bi] > N) continue;
+        const double c = cost_of(M, bns[bi], S_best);
+        if (c < best_cost) best_cost = c, best.BN = bns[bi];
     }
     return best;
 }

@@ -7,7 +7,7 @@
 // bound by the rate and latency with which operand tiles reach an SM, so the
 // kernel is built around latency:
 //   - one CTA per 128 x BN output tile and K range; the K range of a tile is
-//     split over the S CTAs of a thread-block cluster (S = 1, 2, 4 or 8), which
+//     split over the S CTAs of a thread-block cluster (S = 1, 2 or 4), which
 //     keeps 148 SMs busy with 3 row tiles and shortens every CTA's chain of
 //     dependent loads;
 //   - each CTA parks its partial accumulator in its own shared memory; after a
@@ -37,7 +37,8 @@ template <int BN> struct GemmCfg {
     static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
-    static constexpr int MAX_ITEMS = 2;                        // epilogue items whose side inputs are prefetched
+    static constexpr int MAX_ITEMS = BN >= 128 ? 4 : 2;        // epilogue items in flight together per thread
+    static constexpr int MAX_S = 4;                            // largest cluster split
     static constexpr int MIN_CTAS = BN <= 64 ? 2 : 1;
     static_assert(STAGE_BYTES <= RING_BYTES, "staging tile must fit the operand ring");
 };
@@ -54,6 +55,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           int S, Epi epi, L2Prefetch pf, int *status) {
     using G = GemmCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    NFD_TRACE_T0();
     // blockIdx.x = n_tile * S + split; the S splits of a tile form one cluster
     const int split = blockIdx.x % S, n_tile = blockIdx.x / S;
     const int m0 = blockIdx.y * 128, n0 = n_tile * BN;
@@ -105,6 +107,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tma_load_2d(smem_u32(sB + kb * G::B_BYTES), &tmB, full0 + 8 * kb, (kb0 + kb) * 64, n0);
             }
             pdl_wait();
+            NFD_TRACE_MARK(TRK_OTHER + 1);
             for (int kb = 0; kb < pre; ++kb)
                 tma_load_2d(smem_u32(sA + kb * G::A_BYTES), &tmA, full0 + 8 * kb, (kb0 + kb) * 64, m0);
             for (int kb = pre; kb < nkb; ++kb) {
@@ -160,6 +163,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int row = quad * 32 + lane;                    // tile row held by this thread
         if (mbar_wait(accf, 0, status)) {
             tc_fence_after();
+            NFD_TRACE_MARK_T(TRK_OTHER + 2, 64);
             float *srow = stage + (size_t)row * G::SROW;
             constexpr int HC = BN / 2;                       // columns per half
 #pragma unroll
@@ -179,6 +183,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         cluster_sync_all();              // every CTA of the cluster has parked its partial tile
     else
         __syncthreads();
+    NFD_TRACE_MARK_T(TRK_OTHER + 3, 64);
     if (warp >= 2) {
         // sum the S partials in split order, then the fused epilogue: 8 adjacent columns per item
         const uint32_t stage_u32 = smem_u32(stage);
@@ -197,13 +202,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     const float *p = stage + (size_t)trow * G::SROW + cc * 8;
                     v0 = *reinterpret_cast<const float4 *>(p), v1 = *reinterpret_cast<const float4 *>(p + 4);
                 } else {
-                    uint32_t ra = cluster_map(stage_u32 + off, 0);
-                    v0 = ld_cluster_f4(ra), v1 = ld_cluster_f4(ra + 16);
-                    for (int s = 1; s < S; ++s) {
-                        ra = cluster_map(stage_u32 + off, (uint32_t)s);
-                        const float4 u0 = ld_cluster_f4(ra), u1 = ld_cluster_f4(ra + 16);
-                        v0.x += u0.x, v0.y += u0.y, v0.z += u0.z, v0.w += u0.w;
-                        v1.x += u1.x, v1.y += u1.y, v1.z += u1.z, v1.w += u1.w;
+                    // all remote loads first (their latency is long), then the sum in split order
+                    float4 u0[G::MAX_S], u1[G::MAX_S];
+#pragma unroll
+                    for (int s = 0; s < G::MAX_S; ++s) {
+                        if (s < S) {
+                            const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)s);
+                            u0[s] = ld_cluster_f4(ra), u1[s] = ld_cluster_f4(ra + 16);
+                        }
+                    }
+                    v0 = u0[0], v1 = u1[0];
+#pragma unroll
+                    for (int s = 1; s < G::MAX_S; ++s) {
+                        if (s < S) {
+                            v0.x += u0[s].x, v0.y += u0[s].y, v0.z += u0[s].z, v0.w += u0[s].w;
+                            v1.x += u1[s].x, v1.y += u1[s].y, v1.z += u1[s].z, v1.w += u1[s].w;
+                        }
                     }
                 }
                 float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -211,10 +225,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
         }
     }
+    NFD_TRACE_MARK_T(TRK_OTHER + 4, 64);
     tc_fence_before();
-    if (S > 1)
-        cluster_sync_all();              // no CTA leaves while a peer may still read its partial tile
-    else
+    if (S > 1) {
+        cluster_arrive_relaxed();        // no CTA leaves while a peer may still read its partial tile
+        cluster_wait();
+    } else {
         __syncthreads();
+    }
     if (warp == 1) tmem_dealloc(tmem_base, G::TMEM_COLS);
+    NFD_TRACE_END(TRK_GEMM + 16 * (int)(K > 2048) + 32 * (int)(N / 1024));
 }

@@ -11,11 +11,13 @@
 // It does not release its dependents early: a kernel that starts after this one
 // may read the descriptor before its own wait on the predecessor grid.
 __global__ void k_set_params(StepParams p, StepParams *dst) {
+    NFD_TRACE_T0();
     pdl_wait();
     const int n_words = sizeof(StepParams) / 4;
     const int *src = reinterpret_cast<const int *>(&p);
     int *d = reinterpret_cast<int *>(dst);
     for (int i = threadIdx.x; i < n_words; i += blockDim.x) d[i] = src[i];
+    NFD_TRACE_END(TRK_PARAMS);
 }
 
 // ---------------------------------------------------------------------------
@@ -70,6 +72,7 @@ template <typename TS, int MODE>
 __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *const *Wt_l, const TS *const *b_l,
                                               const TS *a_emb, const float *x, float *y, int n_in, int n_out,
                                               size_t y_row_stride, size_t y_layer_stride) {
+    NFD_TRACE_T0();
     pdl_wait();
     pdl_launch();
     constexpr int NV = WVec<TS>::N;
@@ -115,6 +118,7 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
             }
         }
     }
+    NFD_TRACE_END(TRK_GEMV);
 }
 
 // ---------------------------------------------------------------------------
@@ -130,6 +134,7 @@ template <typename TS>
 __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
                                                      float *z) {
     extern __shared__ float s_patch[];          // [PE_TOK][P]
+    NFD_TRACE_T0();
     pdl_wait();
     pdl_launch();
     const int M = sp->nf * D.T;
@@ -185,6 +190,7 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
 #pragma unroll
     for (int t = 0; t < PE_TOK; ++t)
         if (m0 + t < M) z[(size_t)(m0 + t) * D.d + o] = acc[t] + bo;
+    NFD_TRACE_END(TRK_PATCH);
 }
 
 // ---------------------------------------------------------------------------
@@ -208,7 +214,9 @@ template <typename TS>
 __global__ void __launch_bounds__(128) k_adaln(const StepParams *sp, Dims D, const float *z, TS *out,
                                                const float *mod, size_t row_stride, size_t off_shift,
                                                size_t off_scale) {
+    NFD_TRACE_T0();
     pdl_wait();
+    NFD_TRACE_MARK(TRK_OTHER);
     pdl_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m = blockIdx.x * (blockDim.x >> 5) + warp;
@@ -219,11 +227,20 @@ __global__ void __launch_bounds__(128) k_adaln(const StepParams *sp, Dims D, con
     const float *sc = mod + (size_t)row * row_stride + off_scale;
     const float inv_d = 1.0f / (float)D.d;
     if (D.d <= 1024) {
-        float4 v[8];
+        // every load of the row is issued before anything is consumed or stored: z, then shift and scale
+        float4 v[8], a[8], b[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int i = u * 128 + lane * 4;
             v[u] = i < D.d ? *reinterpret_cast<const float4 *>(zr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = u * 128 + lane * 4;
+            if (i < D.d) {
+                a[u] = *reinterpret_cast<const float4 *>(sh + i);
+                b[u] = *reinterpret_cast<const float4 *>(sc + i);
+            }
         }
         float s = 0.f;
 #pragma unroll
@@ -233,22 +250,21 @@ __global__ void __launch_bounds__(128) k_adaln(const StepParams *sp, Dims D, con
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             if (u * 128 + lane * 4 < D.d) {
-                const float a = v[u].x - mean, b = v[u].y - mean, c = v[u].z - mean, e = v[u].w - mean;
-                q += (a * a + b * b) + (c * c + e * e);
+                const float c0 = v[u].x - mean, c1 = v[u].y - mean, c2 = v[u].z - mean, c3 = v[u].w - mean;
+                q += (c0 * c0 + c1 * c1) + (c2 * c2 + c3 * c3);
             }
         }
         const float rstd = rsqrtf(warp_sum(q) * inv_d + D.eps);
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int i = u * 128 + lane * 4;
-            if (i < D.d) {
-                const float4 a = *reinterpret_cast<const float4 *>(sh + i);
-                const float4 b = *reinterpret_cast<const float4 *>(sc + i);
-                store4<TS>(out + (size_t)m * D.d + i, fmaf((v[u].x - mean) * rstd, 1.0f + b.x, a.x),
-                           fmaf((v[u].y - mean) * rstd, 1.0f + b.y, a.y), fmaf((v[u].z - mean) * rstd, 1.0f + b.z, a.z),
-                           fmaf((v[u].w - mean) * rstd, 1.0f + b.w, a.w));
-            }
+            if (i < D.d)
+                store4<TS>(out + (size_t)m * D.d + i, fmaf((v[u].x - mean) * rstd, 1.0f + b[u].x, a[u].x),
+                           fmaf((v[u].y - mean) * rstd, 1.0f + b[u].y, a[u].y),
+                           fmaf((v[u].z - mean) * rstd, 1.0f + b[u].z, a[u].z),
+                           fmaf((v[u].w - mean) * rstd, 1.0f + b[u].w, a[u].w));
         }
+        NFD_TRACE_END(TRK_ADALN);
         return;
     }
     float s = 0.f;
