@@ -68,6 +68,13 @@ struct nfd_ctx {
     FastState fs;
 
     std::vector<int> n_committed, n_tentative;
+    // Deferred commits: the newest n_pending[s] frames of stream s are counted above but their K/V pages are
+    // not written yet; their clean latents, context noise and actions wait in pend_* until the next
+    // speculation carries them along in its first pass (or until something needs the pages).
+    bool lazy = true;
+    std::vector<int> n_pending;
+    std::vector<std::vector<int>> pend_act;
+    float *pend_x0 = nullptr, *pend_cz = nullptr;     // [n_streams][k_max][C,H,W]
     // Modulation cache: the adaLN modulation depends on (FM time, action) only, so each pair is computed
     // once and kept in one of n_slots rows of `mod` / `fmod`; least recently used rows are replaced.
     struct CondSlot {
@@ -415,7 +422,76 @@ static int run_pass_inner(nfd_ctx *c) {
     return NFD_OK;
 }
 
-// Fill c->h_sp for a pass over n streams x k frames.
+// One frame of a pass as the host describes it.
+struct PassFrame {
+    int stream, frame;       // batch slot, absolute frame index
+    float t;                 // FM time
+    int action;
+    int first_new;           // first frame of the stream whose K/V this pass writes
+    int src, src_index;      // input set and frame slot in it
+    int out_index;           // v_out slot or -1
+};
+
+struct PassInputs {
+    const float *x_a[2] = {nullptr, nullptr}, *x_b[2] = {nullptr, nullptr};
+    float alpha[2] = {0.f, 0.f}, beta[2] = {0.f, 0.f};
+    float *v_out = nullptr;
+};
+
+// Fill c->h_sp for a pass over the given frames.  Nothing is changed if it fails.
+static int build_pass_frames(nfd_ctx *c, const std::vector<PassFrame> &fr, int kind, const PassInputs &in) {
+    const nfd_cfg &g = c->cfg;
+    const int nf = (int)fr.size();
+    if (nf < 1 || nf > NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;
+    // validate everything before the modulation cache is touched
+    for (const PassFrame &f : fr) {
+        if (f.stream < 0 || f.stream >= g.n_streams) return NFD_E_RANGE;
+        if (!(f.t >= 0.f) || !(f.t <= 1.f)) return NFD_E_RANGE;
+        if (f.action < 0 || f.action >= g.n_actions) return NFD_E_RANGE;
+    }
+    StepParams &p = c->h_sp;
+    memset(&p, 0, sizeof(p));
+    ++c->pass_no;
+    p.nf = nf;
+    p.kind = kind;
+    for (int s = 0; s < 2; ++s) p.x_a[s] = in.x_a[s], p.x_b[s] = in.x_b[s], p.alpha[s] = in.alpha[s], p.beta[s] = in.beta[s];
+    p.v_out = in.v_out;
+    int nc = 0;
+    for (int j = 0; j < nf; ++j) {
+        const PassFrame &pf = fr[j];
+        // modulation cache: reuse the slot of this (t, action) pair, else take the least recently used one
+        unsigned tb;
+        memcpy(&tb, &pf.t, 4);
+        int row = -1, lru = -1;
+        for (int r = 0; r < (int)c->cond_slots.size(); ++r) {
+            const nfd_ctx::CondSlot &cs = c->cond_slots[r];
+            if (cs.action == pf.action && cs.t_bits == tb) row = r;
+            if (cs.last_use != c->pass_no && (lru < 0 || cs.last_use < c->cond_slots[lru].last_use)) lru = r;
+        }
+        if (row < 0) {
+            if (lru < 0 || nc >= NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;      // cannot happen: slots > frames per pass
+            row = lru;
+            c->cond_slots[row].t_bits = tb, c->cond_slots[row].action = pf.action;
+            p.cd[nc].t = pf.t, p.cd[nc].action = pf.action, p.cd[nc].slot = row;
+            ++nc;
+            ++c->cond_misses;
+        } else if (c->cond_slots[row].last_use != c->pass_no) {
+            ++c->cond_hits;
+        }
+        c->cond_slots[row].last_use = c->pass_no;
+        FrameDesc &f = p.fr[j];
+        f.stream = pf.stream;
+        f.frame = pf.frame;
+        f.win_first = pf.frame - g.ctx_frames > 0 ? pf.frame - g.ctx_frames : 0;
+        f.cond_row = row;
+        f.first_new = pf.first_new;
+        f.src = pf.src, f.src_index = pf.src_index, f.out_index = pf.out_index;
+    }
+    p.nc = nc;
+    return NFD_OK;
+}
+
+// A pass over n streams x k frames that follow the frames counted so far (plus `offset`).
 //   actions: per stream (per_frame_actions = false) or per frame.
 static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, const float *t, const int *actions,
                       bool per_frame_actions, int kind, const float *x_a, float alpha, const float *x_b, float beta,
@@ -428,54 +504,21 @@ static int build_pass(nfd_ctx *c, int n, const int *streams, int k, int offset, 
         for (int j = 0; j < i; ++j)
             if (streams[j] == streams[i]) return NFD_E_RANGE;
     }
-    // validate everything before the modulation cache is touched: a failed call changes nothing
-    for (int i = 0; i < n; ++i) {
-        if (!(t[i] >= 0.f) || !(t[i] <= 1.f)) return NFD_E_RANGE;
-        for (int j = 0; j < (per_frame_actions ? k : 1); ++j) {
-            const int a = per_frame_actions ? actions[i * k + j] : actions[i];
-            if (a < 0 || a >= g.n_actions) return NFD_E_RANGE;
-        }
-    }
-    StepParams &p = c->h_sp;
-    memset(&p, 0, sizeof(p));
-    ++c->pass_no;
-    p.nf = n * k;
-    p.kind = kind;
-    p.x_a = x_a, p.x_b = x_b, p.alpha = alpha, p.beta = beta, p.v_out = v_out;
-    int nc = 0;
-    for (int i = 0; i < n; ++i) {
+    std::vector<PassFrame> fr;
+    for (int i = 0; i < n; ++i)
         for (int j = 0; j < k; ++j) {
-            int a = per_frame_actions ? actions[i * k + j] : actions[i];
-            // modulation cache: reuse the slot of this (t, action) pair, else take the least recently used one
-            unsigned tb;
-            memcpy(&tb, &t[i], 4);
-            int row = -1, lru = -1;
-            for (int r = 0; r < (int)c->cond_slots.size(); ++r) {
-                const nfd_ctx::CondSlot &cs = c->cond_slots[r];
-                if (cs.action == a && cs.t_bits == tb) row = r;
-                if (cs.last_use != c->pass_no && (lru < 0 || cs.last_use < c->cond_slots[lru].last_use)) lru = r;
-            }
-            if (row < 0) {
-                if (lru < 0 || nc >= NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;      // cannot happen: slots > frames per pass
-                row = lru;
-                c->cond_slots[row].t_bits = tb, c->cond_slots[row].action = a;
-                p.cd[nc].t = t[i], p.cd[nc].action = a, p.cd[nc].slot = row;
-                ++nc;
-                ++c->cond_misses;
-            } else if (c->cond_slots[row].last_use != c->pass_no) {
-                ++c->cond_hits;
-            }
-            c->cond_slots[row].last_use = c->pass_no;
-            FrameDesc &f = p.fr[i * k + j];
+            PassFrame f;
             f.stream = streams[i];
             f.frame = c->n_total(streams[i]) + offset + j;
-            f.win_first = f.frame - g.ctx_frames > 0 ? f.frame - g.ctx_frames : 0;
-            f.cond_row = row;
+            f.t = t[i];
+            f.action = per_frame_actions ? actions[i * k + j] : actions[i];
             f.first_new = c->n_total(streams[i]) + offset;
+            f.src = 0, f.src_index = i * k + j, f.out_index = i * k + j;
+            fr.push_back(f);
         }
-    }
-    p.nc = nc;
-    return NFD_OK;
+    PassInputs in;
+    in.x_a[0] = x_a, in.x_b[0] = x_b, in.alpha[0] = alpha, in.beta[0] = beta, in.v_out = v_out;
+    return build_pass_frames(c, fr, kind, in);
 }
 
 // ---------------------------------------------------------------------------
@@ -527,11 +570,14 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     D.L = cfg->n_layers, D.d = cfg->d_model, D.H = cfg->n_heads, D.dh = cfg->head_dim, D.dm = cfg->d_mlp;
     D.C = cfg->latent_c, D.Hl = cfg->latent_h, D.Wl = cfg->latent_w, D.p = cfg->patch;
     D.th = D.Hl / D.p, D.tw = D.Wl / D.p, D.T = D.th * D.tw, D.P = D.C * D.p * D.p;
-    D.R = cfg->ctx_frames + cfg->max_spec, D.W = cfg->ctx_frames, D.n_streams = cfg->n_streams;
+    // ring pages per layer: the window, the frames of a speculation and the deferred frames that may ride along
+    D.R = cfg->ctx_frames + 2 * cfg->max_spec, D.W = cfg->ctx_frames, D.n_streams = cfg->n_streams;
     D.norm = cfg->norm, D.eps = cfg->norm_eps, D.t_scale = cfg->t_scale;
     D.page_elems = (size_t)D.H * D.T * D.dh;
     c->n_committed.assign(cfg->n_streams, 0);
     c->n_tentative.assign(cfg->n_streams, 0);
+    c->n_pending.assign(cfg->n_streams, 0);
+    c->pend_act.assign(cfg->n_streams, std::vector<int>());
     if (getenv("NFD_NO_GRAPH")) c->use_graph = false;
     if (getenv("NFD_NO_FAST")) c->fast = false;
 
@@ -554,6 +600,8 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     c->cond_slots.assign(n_slots, nfd_ctx::CondSlot());
     A((void **)&c->mod, (size_t)n_slots * D.L * 6 * D.d * 4);
     A((void **)&c->fmod, (size_t)n_slots * 2 * D.d * 4);
+    A((void **)&c->pend_x0, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);
+    A((void **)&c->pend_cz, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);
     A((void **)&c->xp, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->vbuf, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->d_sp, sizeof(StepParams));
@@ -603,8 +651,11 @@ int nfd_reset(nfd_ctx *c, int stream) {
     if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
     c->n_committed[stream] = 0;
     c->n_tentative[stream] = 0;
+    c->n_pending[stream] = 0;
     return NFD_OK;
 }
+
+static int flush_pending(nfd_ctx *c, int s);
 
 static int check_io(const void *a, const void *b) {
     if (!a || !b) return NFD_E_NULLPTR;
@@ -616,6 +667,10 @@ int nfd_denoise_step_batched(nfd_ctx *c, int n, const int *streams, const float 
                              const int *actions, float *v_out) {
     if (!c || !streams || !t || !actions) return NFD_E_NULLPTR;
     RET(check_io(x_t, v_out));
+    for (int i = 0; i < n; ++i) {
+        if (streams[i] < 0 || streams[i] >= c->cfg.n_streams) return NFD_E_RANGE;
+        RET(flush_pending(c, streams[i]));
+    }
     RET(build_pass(c, n, streams, k, 0, t, actions, false, 0, x_t, 1.0f, nullptr, 0.f, v_out));
     return run_pass(c);
 }
@@ -624,6 +679,9 @@ int nfd_denoise_step_at(nfd_ctx *c, int stream, int offset, const float *x_t, in
                         float *v_out) {
     if (!c) return NFD_E_NULLPTR;
     RET(check_io(x_t, v_out));
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    if (!(t >= 0.f) || !(t <= 1.f) || action < 0 || action >= c->cfg.n_actions) return NFD_E_RANGE;
+    RET(flush_pending(c, stream));
     RET(build_pass(c, 1, &stream, k, offset, &t, &action, false, 0, x_t, 1.0f, nullptr, 0.f, v_out));
     return run_pass(c);
 }
@@ -632,18 +690,54 @@ int nfd_denoise_step(nfd_ctx *c, int stream, const float *x_t, int k, float t, i
     return nfd_denoise_step_at(c, stream, 0, x_t, k, t, action, v_out);
 }
 
+// Input scaling of a commit (Section 4.3): x' = cos(t_ctx) x0 + sin(t_ctx) sigma_d z at the constant context
+// timestep, then brought to Flow-Matching scale; returns the FM time and the two coefficients.
+static void commit_coeffs(const nfd_ctx *c, float *t_fm, float *a, float *b) {
+    const double tc = c->cfg.t_ctx_trig, sd = c->cfg.sigma_d;
+    const double sn = sin(tc), cs = cos(tc);
+    const double t = sn / (sn + cs);
+    const double scale = sqrt(t * t + (1 - t) * (1 - t));
+    *t_fm = (float)t, *a = (float)(cs * scale / sd), *b = (float)(sn * scale);
+}
+
 // Commit pass over n streams x k frames; actions per frame.
 static int commit_pass(nfd_ctx *c, int n, const int *streams, int k, const int *actions, const float *x0,
                        const float *ctx_noise, bool tentative) {
-    const double tc = c->cfg.t_ctx_trig, sd = c->cfg.sigma_d;
-    const double sn = sin(tc), cs = cos(tc);
-    const double t_fm = sn / (sn + cs);
-    const double scale = sqrt(t_fm * t_fm + (1 - t_fm) * (1 - t_fm));
-    std::vector<float> t(n, (float)t_fm);
-    RET(build_pass(c, n, streams, k, 0, t.data(), actions, true, 1, x0, (float)(cs * scale / sd), ctx_noise,
-                   (float)(sn * scale), nullptr));
+    float t_fm, ca, cb;
+    commit_coeffs(c, &t_fm, &ca, &cb);
+    std::vector<float> t(n, t_fm);
+    RET(build_pass(c, n, streams, k, 0, t.data(), actions, true, 1, x0, ca, ctx_noise, cb, nullptr));
     RET(run_pass(c));
     for (int i = 0; i < n; ++i) (tentative ? c->n_tentative : c->n_committed)[streams[i]] += k;
+    return NFD_OK;
+}
+
+// Frames of stream s whose commit was deferred, as frames of a pass (input set `set`, K/V only).
+static void pending_frames(const nfd_ctx *c, int s, int set, std::vector<PassFrame> &fr) {
+    float t_fm, ca, cb;
+    commit_coeffs(c, &t_fm, &ca, &cb);
+    const int P = c->n_pending[s], total = c->n_total(s);
+    for (int j = 0; j < P; ++j) {
+        PassFrame f;
+        f.stream = s, f.frame = total - P + j, f.t = t_fm, f.action = c->pend_act[s][j];
+        f.first_new = total - P;
+        f.src = set, f.src_index = s * c->cfg.max_spec + j, f.out_index = -1;
+        fr.push_back(f);
+    }
+}
+
+// Write the K/V pages of the deferred frames of one stream now (a commit pass of their own).
+static int flush_pending(nfd_ctx *c, int s) {
+    if (c->n_pending[s] == 0) return NFD_OK;
+    std::vector<PassFrame> fr;
+    pending_frames(c, s, 0, fr);
+    PassInputs in;
+    float t_fm;
+    commit_coeffs(c, &t_fm, &in.alpha[0], &in.beta[0]);
+    in.x_a[0] = c->pend_x0, in.x_b[0] = c->pend_cz;
+    RET(build_pass_frames(c, fr, 1, in));
+    RET(run_pass(c));
+    c->n_pending[s] = 0;
     return NFD_OK;
 }
 
@@ -652,6 +746,10 @@ int nfd_commit_frame(nfd_ctx *c, int stream, const float *x0, int n, const int *
     if (!aligned16(x0) || !aligned16(ctx_noise)) return NFD_E_ALIGN;
     if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
     if (c->n_tentative[stream] != 0) return NFD_E_STATE;
+    if (n < 1 || n > c->cfg.max_spec) return NFD_E_RANGE;
+    for (int j = 0; j < n; ++j)
+        if (actions[j] < 0 || actions[j] >= c->cfg.n_actions) return NFD_E_RANGE;
+    RET(flush_pending(c, stream));
     return commit_pass(c, 1, &stream, n, actions, x0, ctx_noise, false);
 }
 
@@ -661,14 +759,23 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
     RET(check_io(noise, x0_out));
     if (!aligned16(ctx_noise)) return NFD_E_ALIGN;
     if (n < 1 || k < 1 || k > c->cfg.max_spec || (long long)n * k > NFD_MAX_PASS_FRAMES) return NFD_E_RANGE;
+    int n_pend = 0;
     for (int i = 0; i < n; ++i) {
         if (streams[i] < 0 || streams[i] >= c->cfg.n_streams) return NFD_E_RANGE;
+        for (int j = 0; j < i; ++j)
+            if (streams[j] == streams[i]) return NFD_E_RANGE;
         if (actions[i] < 0 || actions[i] >= c->cfg.n_actions) return NFD_E_RANGE;
         if (c->n_tentative[streams[i]] != 0) return NFD_E_STATE;
+        n_pend += c->n_pending[streams[i]];
     }
+    // deferred frames ride along with the first denoising pass if the pass can hold them
+    const bool carry = c->lazy && n_pend > 0 && n * k + n_pend <= NFD_MAX_PASS_FRAMES;
+    if (!carry)
+        for (int i = 0; i < n; ++i) RET(flush_pending(c, streams[i]));
     const int S = c->cfg.n_steps;
     const double sd = c->cfg.sigma_d;
-    const size_t ne = (size_t)n * k * c->frame_elems();
+    const size_t fe = c->frame_elems();
+    const size_t ne = (size_t)n * k * fe;
     const int eg = (int)((ne + 255) / 256);
     // Section 4.1 "Sampling": start from pure noise at t' = pi/2
     c->cls = CLS_SAMPLER;
@@ -680,9 +787,33 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
         const double t = sn / (sn + cs);
         const double alpha = sqrt(t * t + (1 - t) * (1 - t)) / sd;
         for (int i = 0; i < n; ++i) tv[i] = (float)t;
-        RET(build_pass(c, n, streams, k, 0, tv.data(), actions, false, 0, c->xp, (float)alpha, nullptr, 0.f,
-                       c->vbuf));
-        RET(run_pass(c));
+        if (s == 0 && carry) {
+            // one block-causal pass: per stream its deferred frames (K/V only), then the k new frames
+            std::vector<PassFrame> fr;
+            for (int i = 0; i < n; ++i) {
+                const int st = streams[i], total = c->n_total(st), P = c->n_pending[st];
+                pending_frames(c, st, 1, fr);
+                for (int j = 0; j < k; ++j) {
+                    PassFrame f;
+                    f.stream = st, f.frame = total + j, f.t = (float)t, f.action = actions[i];
+                    f.first_new = total - P;
+                    f.src = 0, f.src_index = i * k + j, f.out_index = i * k + j;
+                    fr.push_back(f);
+                }
+            }
+            PassInputs in;
+            float t_fm;
+            commit_coeffs(c, &t_fm, &in.alpha[1], &in.beta[1]);
+            in.x_a[1] = c->pend_x0, in.x_b[1] = c->pend_cz;
+            in.x_a[0] = c->xp, in.alpha[0] = (float)alpha, in.v_out = c->vbuf;
+            RET(build_pass_frames(c, fr, 0, in));
+            RET(run_pass(c));
+            for (int i = 0; i < n; ++i) c->n_pending[streams[i]] = 0;
+        } else {
+            RET(build_pass(c, n, streams, k, 0, tv.data(), actions, false, 0, c->xp, (float)alpha, nullptr, 0.f,
+                           c->vbuf));
+            RET(run_pass(c));
+        }
         // clean estimate sigma_d (x_in - t v), then re-noise to the next timestep
         const float *z = nullptr;
         double cn = 0, sn_next = 0;
@@ -696,10 +827,29 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
                 (float)(-sd * t), (float)cn, (float)sn_next, ne);
     }
     CK(cudaGetLastError());
-    std::vector<int> fa((size_t)n * k);
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < k; ++j) fa[i * k + j] = actions[i];
-    return commit_pass(c, n, streams, k, fa.data(), x0_out, ctx_noise, true);
+    CK(c->launch_err);
+    if (!c->lazy) {
+        std::vector<int> fa((size_t)n * k);
+        for (int i = 0; i < n; ++i)
+            for (int j = 0; j < k; ++j) fa[i * k + j] = actions[i];
+        return commit_pass(c, n, streams, k, fa.data(), x0_out, ctx_noise, true);
+    }
+    // defer the commit: keep what it needs; the frames count as tentative from now on
+    for (int i = 0; i < n; ++i) {
+        const int st = streams[i];
+        const size_t off = (size_t)st * c->cfg.max_spec * fe;
+        CK(cudaMemcpyAsync(c->pend_x0 + off, x0_out + (size_t)i * k * fe, (size_t)k * fe * 4, cudaMemcpyDeviceToDevice,
+                           c->st));
+        if (ctx_noise)
+            CK(cudaMemcpyAsync(c->pend_cz + off, ctx_noise + (size_t)i * k * fe, (size_t)k * fe * 4,
+                               cudaMemcpyDeviceToDevice, c->st));
+        else
+            CK(cudaMemsetAsync(c->pend_cz + off, 0, (size_t)k * fe * 4, c->st));
+        c->pend_act[st].assign(k, actions[i]);
+        c->n_pending[st] = k;
+        c->n_tentative[st] += k;
+    }
+    return NFD_OK;
 }
 
 int nfd_speculate(nfd_ctx *c, int stream, int k, int action, const float *noise, const float *ctx_noise,
@@ -713,6 +863,7 @@ int nfd_rollback(nfd_ctx *c, int stream, int n_accept) {
     if (n_accept < 0 || n_accept > c->n_tentative[stream]) return NFD_E_RANGE;
     c->n_committed[stream] += n_accept;
     c->n_tentative[stream] = 0;
+    if (c->n_pending[stream] > n_accept) c->n_pending[stream] = n_accept;     // rejected frames were never written
     return NFD_OK;
 }
 
@@ -729,6 +880,7 @@ int nfd_kv_state(nfd_ctx *c, int stream, int *n_committed, int *n_tentative, int
 int nfd_kv_hash(nfd_ctx *c, int stream, unsigned long long *h) {
     if (!c || !h) return NFD_E_NULLPTR;
     if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    RET(flush_pending(c, stream));
     const int total = c->n_total(stream);
     const int first = total - c->cfg.ctx_frames > 0 ? total - c->cfg.ctx_frames : 0;
     const int count = total - first;
@@ -755,6 +907,7 @@ int nfd_kv_hash(nfd_ctx *c, int stream, unsigned long long *h) {
 int nfd_kv_read(nfd_ctx *c, int stream, int layer, int frame, float *k_out, float *v_out) {
     if (!c) return NFD_E_NULLPTR;
     if (stream < 0 || stream >= c->cfg.n_streams || layer < 0 || layer >= c->cfg.n_layers) return NFD_E_RANGE;
+    RET(flush_pending(c, stream));
     const int total = c->n_total(stream);
     if (frame < 0 || frame >= total + c->cfg.max_spec || frame < total + c->cfg.max_spec - c->D.R) return NFD_E_RANGE;
     const int grid = (int)((c->D.page_elems + 255) / 256);
@@ -782,6 +935,7 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
     const Dims &D = c->D;
     c->n_committed[0] = 0;
     c->n_tentative[0] = 0;
+    c->n_pending[0] = 0;
     const size_t fill = (size_t)n_kv * D.page_elems;
     c->cls = CLS_CACHE;
     if (k) {
@@ -870,6 +1024,12 @@ int nfd_set_option(nfd_ctx *c, const char *name, int value) {
     }
     if (!strcmp(name, "fast")) {
         c->fast = value != 0;
+        return NFD_OK;
+    }
+    if (!strcmp(name, "lazy_commit")) {
+        if (!value)
+            for (int s = 0; s < c->cfg.n_streams; ++s) RET(flush_pending(c, s));
+        c->lazy = value != 0;
         return NFD_OK;
     }
     return NFD_E_RANGE;

@@ -14,6 +14,9 @@ struct FrameDesc {
     int win_first;   // first frame this one attends to (>= 0, >= frame - W)
     int cond_row;    // slot of the modulation cache that holds this frame's adaLN modulation
     int first_new;   // first frame of this stream whose K/V the current pass writes (earlier pages are final)
+    int src;         // which input set of the pass this frame's latent comes from (0 or 1)
+    int src_index;   // frame slot inside that input set
+    int out_index;   // frame slot of v_out this frame's velocity goes to, or -1 (no output wanted)
 };
 
 // One (FM time, action) pair whose modulation this pass has to compute: the pairs
@@ -32,10 +35,13 @@ struct StepParams {
     int nc;                 // conditioning rows to compute in this pass (0: every pair is cached)
     int kind;               // 0 denoise (all layers + velocity head), 1 commit (K/V only)
     int layer_for_attn;     // nfd_attention: which layer's pages hold the data
-    const float *x_a;       // model input = alpha * x_a + beta * x_b
-    const float *x_b;       // may be NULL
-    float *v_out;           // [nf,C,H,W]
-    float alpha, beta;
+    // Two input sets: a frame's model input is alpha[s] * x_a[s] + beta[s] * x_b[s] with s = its `src`.
+    // Set 0 feeds the frames being denoised (or committed), set 1 the frames whose commit was deferred
+    // and rides along with this pass.
+    const float *x_a[2];
+    const float *x_b[2];    // may be NULL
+    float alpha[2], beta[2];
+    float *v_out;           // [frames with out_index >= 0, C,H,W]
     FrameDesc fr[NFD_MAX_PASS_FRAMES];
     CondDesc cd[NFD_MAX_PASS_FRAMES];
 };

@@ -140,8 +140,6 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
     const int M = sp->nf * D.T;
     const int m0 = blockIdx.x * PE_TOK;
     if (m0 >= M) return;
-    const float *xa = sp->x_a, *xb = sp->x_b;
-    const float alpha = sp->alpha, beta = sp->beta;
     for (int i = threadIdx.x; i < PE_TOK * D.P; i += blockDim.x) {
         const int t = i / D.P, p = i - t * D.P, m = m0 + t;
         float v = 0.f;
@@ -149,9 +147,11 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
             const int j = m / D.T, tok = m % D.T;
             const int r = tok / D.tw, c = tok % D.tw;
             const int ch = p / (D.p * D.p), py = (p / D.p) % D.p, px = p % D.p;
-            const size_t idx = (((size_t)j * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
-            v = alpha * xa[idx];
-            if (xb) v = fmaf(beta, xb[idx], v);
+            const int set = sp->fr[j].src, fj = sp->fr[j].src_index;
+            const float *xa = sp->x_a[set], *xb = sp->x_b[set];
+            const size_t idx = (((size_t)fj * D.C + ch) * D.Hl + (r * D.p + py)) * D.Wl + (c * D.p + px);
+            v = sp->alpha[set] * xa[idx];
+            if (xb) v = fmaf(sp->beta[set], xb[idx], v);
         }
         s_patch[i] = v;
     }
@@ -502,7 +502,9 @@ template <typename TS> struct EpiFinal {
         for (int i = 0; i < 8; i += 2) (*this)(m, n + i, a[i], a[i + 1]);
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
-        const int j = m / D.T, tok = m % D.T;
+        const int jp = m / D.T, tok = m % D.T;
+        const int j = sp->fr[jp].out_index;        // frames that only ride along for their K/V have no output
+        if (j < 0) return;
         const int r = tok / D.tw, c = tok % D.tw;
         float av[2] = {a0 + to_f(bias[n]), a1 + to_f(bias[n + 1])};
 #pragma unroll

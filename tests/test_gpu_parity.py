@@ -306,3 +306,41 @@ def test_modulation_cache_hits_evictions_and_values():
         g.denoise_step(x, 0.3333, 99)
     assert g.cond_cache_stats() == (h1, m1 + 1)
     assert g.status() == 0
+
+
+@pytest.mark.parametrize("name", ["tiny_bf16", "tiny", "nfd310m_slice"])
+def test_deferred_commit_equals_immediate_commit(name):
+    """A speculation leaves the commit of its frames to the first pass of the next speculation (the paper's
+    "compute and cache their KVs during the first denoising step", Appendix on KV caching).  Frames, counters
+    and cache contents must be bitwise those of a context that commits at once, whatever mix of k and
+    accepted counts is used, and whatever call forces the deferred pages to be written."""
+    from paper_2506_01380_b200.nfd import NFD
+    torch = _torch()
+    cfg = I.make_cfg(name)
+    w = I.make_weights(cfg, 7, "stress")
+    lazy, eager = NFD(cfg, w), NFD(cfg, w)
+    eager.set_option("lazy_commit", 0)
+    x0 = dev(I.make_latents(cfg, 2, 11))
+    for g in (lazy, eager):
+        g.commit_frame(x0, [1, 2], dev(I.make_latents(cfg, 2, 12)))
+    S = cfg["n_steps"]
+    plan = [(2, 1), (1, 1), (3, 3), (4, 2), (1, 1), (2, 2)]          # (k, accepted)
+    for step, (k, n_acc) in enumerate(plan):
+        noise = dev(I.make_noise(cfg, S, k, 100 + step))
+        cz = dev(I.make_latents(cfg, k, 200 + step)) if step % 2 == 0 else None
+        ya = lazy.speculate(k, step % cfg["n_actions"], noise, cz)
+        yb = eager.speculate(k, step % cfg["n_actions"], noise, cz)
+        assert torch.equal(ya, yb), f"speculation {step}: frames differ"
+        assert lazy.kv_state() == eager.kv_state()
+        lazy.rollback(n_acc)
+        eager.rollback(n_acc)
+        assert lazy.kv_state() == eager.kv_state()
+        if step == 3:                                                 # forces the deferred pages out mid-way
+            assert lazy.kv_hash() == eager.kv_hash()
+    assert lazy.kv_hash() == eager.kv_hash()
+    L, total = cfg["n_layers"], lazy.kv_state()[0]
+    for f in (total - 1, total - 2):
+        Ka, Va = lazy.kv_read(L - 1, f)
+        Kb, Vb = eager.kv_read(L - 1, f)
+        assert torch.equal(Ka, Kb) and torch.equal(Va, Vb)
+    assert lazy.status() == 0 and eager.status() == 0
