@@ -143,9 +143,11 @@ struct GemmPlan {
     int BN, S;
 };
 
-// CTAs that can be resident at once: two per SM for the narrow tiles (their shared
-// memory is sized for that), one for the wide ones.
-static int gemm_slots(int n_sm, int BN) { return BN <= 64 ? 2 * n_sm : n_sm; }
+// CTAs that can be resident at once: one per SM.
+static int gemm_slots(int n_sm, int BN) {
+    (void)BN;
+    return n_sm;
+}
 
 static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind) {
     // optional override for tuning: NFD_GEMM_PLAN="kind:BN:S,kind:BN:S,..." (kind = TC_* value, +10 for K > 2048)
@@ -168,19 +170,19 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
         const long long ctas = (long long)mt * nt * S;
         const int slots = gemm_slots(fs.n_sm, BN);
         const double waves = (double)((ctas + slots - 1) / slots);
-        const double share = ctas > fs.n_sm ? (double)(ctas < slots ? ctas : slots) / fs.n_sm : 1.0;
+        const double share = 1.0;
         const double kb = (double)((nkb + S - 1) / S);
         const double load = kb * (16384.0 + BN * 128.0) / 55.0 * share;
         const double items = (128.0 / S) * (BN / 8.0) / 256.0;                 // epilogue items per thread
-        const double epi = 400.0 + items * (S > 1 ? 700.0 : 350.0) + BN * 4.0;
-        const double fixed = 3200.0 + (S > 1 ? 1500.0 : 0.0);
+        const double epi = 400.0 + items * 350.0 + (S - 1) * 900.0 + BN * 4.0;     // remote partials are slow to fetch
+        const double fixed = 3200.0 + (S > 1 ? 800.0 : 0.0);
         return waves * (fixed + load + epi);
     };
-    const int bns[3] = {32, 64, 128};
+    const int bns[4] = {32, 64, 96, 128};
     const int T = (int)(fs.a_rows / NFD_MAX_PASS_FRAMES);
     int S_best = 1;
     double best_cost = 1e30;
-    for (int bi = 0; bi < 3; ++bi) {
+    for (int bi = 0; bi < 4; ++bi) {
         if (bns[bi] > 32 && bns[bi] > N) continue;
         for (int S = 1; S <= GemmCfg<64>::MAX_S; S *= 2) {
             if (S > 1 && nkb / S < 2) break;
@@ -190,7 +192,7 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
     }
     GemmPlan best{32, S_best};
     best_cost = 1e30;
-    for (int bi = 0; bi < 3; ++bi) {
+    for (int bi = 0; bi < 4; ++bi) {
         if (bns[bi] > 32 && bns[bi] > N) continue;
         const double c = cost_of(M, bns[bi], S_best);
         if (c < best_cost) best_cost = c, best.BN = bns[bi];
@@ -237,6 +239,7 @@ static bool fast_gemm(bool enabled, FastState &fs, cudaStream_t st, const TS *A,
         const GemmPlan pl = plan_gemm(fs, M, N, K, tc_kind);
         switch (pl.BN) {
             case 128: return launch_gemm_tc<128, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
+            case 96: return launch_gemm_tc<96, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
             case 64: return launch_gemm_tc<64, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
             default: return launch_gemm_tc<32, Epi>(fs, st, A, Wt, M, N, K, pl.S, epi, pf);
         }

@@ -23,11 +23,15 @@
 //     (bias, gate, residual, rotary table) are fetched while the UMMAs run;
 //   - every CTA also pulls a slice of the NEXT GEMM's weights towards L2, so that
 //     the weight stream from HBM runs one kernel ahead of its use.
+// One CTA fills an SM (its operand ring is sized for that): with programmatic
+// dependent launch CTAs are placed wherever there is room at that moment, and
+// two small CTAs piling onto one SM while others stay empty costs more than it
+// gains.
 #pragma once
 #include "nfd_sm100.cuh"
 
 template <int BN> struct GemmCfg {
-    static constexpr int STAGES = BN <= 64 ? 4 : 6;
+    static constexpr int STAGES = BN <= 32 ? 7 : 6;             // ring deep enough that one CTA owns an SM
     static constexpr int A_BYTES = 128 * 128;                  // 128 rows x 64 bf16
     static constexpr int B_BYTES = BN * 128;
     static constexpr int RING_BYTES = STAGES * (A_BYTES + B_BYTES);
@@ -37,9 +41,9 @@ template <int BN> struct GemmCfg {
     static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
-    static constexpr int MAX_ITEMS = BN >= 128 ? 4 : 2;        // epilogue items in flight together per thread
+    static constexpr int MAX_ITEMS = 4;                        // epilogue items in flight together per thread
     static constexpr int MAX_S = 4;                            // largest cluster split
-    static constexpr int MIN_CTAS = BN <= 64 ? 2 : 1;
+    static constexpr int MIN_CTAS = 1;
     static_assert(STAGE_BYTES <= RING_BYTES, "staging tile must fit the operand ring");
 };
 
@@ -137,6 +141,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 const int s = kb % G::STAGES;
                 if (!mbar_wait(full0 + 8 * s, (kb / G::STAGES) & 1, status)) break;
                 tc_fence_after();
+                if (kb == 0) NFD_TRACE_MARK_T(TRK_OTHER + 5, 32);
+                if (kb == nkb - 1) NFD_TRACE_MARK_T(TRK_OTHER + 6, 32);
                 const uint64_t ad = umma_desc_k128(smem_u32(sA + s * G::A_BYTES));
                 const uint64_t bd = umma_desc_k128(smem_u32(sB + s * G::B_BYTES));
 #pragma unroll
