@@ -41,7 +41,7 @@ template <int BN> struct GemmCfg {
     static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
-    static constexpr int MAX_ITEMS = 4;                        // epilogue items in flight together per thread
+    static constexpr int MAX_ITEMS = 2;                        // epilogue items in flight together per thread
     static constexpr int MAX_S = 4;                            // largest cluster split
     static constexpr int MIN_CTAS = 1;
     static_assert(STAGE_BYTES <= RING_BYTES, "staging tile must fit the operand ring");
@@ -191,43 +191,50 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __syncthreads();
     NFD_TRACE_MARK_T(TRK_OTHER + 3, 64);
     if (warp >= 2) {
-        // sum the S partials in split order, then the fused epilogue: 8 adjacent columns per item
+        // Items in batches of MAX_ITEMS.  Phase A issues every load of the batch (side inputs, and the S
+        // partials, remote ones through distributed shared memory: their latency is long); phase B sums the
+        // partials in split order and runs the fused epilogue, 8 adjacent columns per item.
         const uint32_t stage_u32 = smem_u32(stage);
         for (int i0 = 0; i0 * G::EPI_THREADS < n_items; i0 += G::MAX_ITEMS) {
+            float4 u0[G::MAX_ITEMS][G::MAX_S], u1[G::MAX_ITEMS][G::MAX_S];
+            int mm[G::MAX_ITEMS], nn[G::MAX_ITEMS];
 #pragma unroll
             for (int i = 0; i < G::MAX_ITEMS; ++i) {
                 const int it = et + (i0 + i) * G::EPI_THREADS;
-                if (it >= n_items) continue;
                 const int trow = r_base + it / CPR, cc = it % CPR;
-                const int m = m0 + trow, n = n0 + cc * 8;
-                if (m >= M || n >= N) continue;
-                if (i0 > 0) epi.load(m, n, side[i]);
+                mm[i] = m0 + trow, nn[i] = n0 + cc * 8;
+                if (it >= n_items || mm[i] >= M || nn[i] >= N) {
+                    mm[i] = -1;
+                    continue;
+                }
+                if (i0 > 0) epi.load(mm[i], nn[i], side[i]);
                 const uint32_t off = (uint32_t)(trow * G::SROW + cc * 8) * 4;
-                float4 v0, v1;
                 if (S == 1) {
                     const float *p = stage + (size_t)trow * G::SROW + cc * 8;
-                    v0 = *reinterpret_cast<const float4 *>(p), v1 = *reinterpret_cast<const float4 *>(p + 4);
+                    u0[i][0] = *reinterpret_cast<const float4 *>(p), u1[i][0] = *reinterpret_cast<const float4 *>(p + 4);
                 } else {
-                    // all remote loads first (their latency is long), then the sum in split order
-                    float4 u0[G::MAX_S], u1[G::MAX_S];
 #pragma unroll
-                    for (int s = 0; s < G::MAX_S; ++s) {
-                        if (s < S) {
-                            const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)s);
-                            u0[s] = ld_cluster_f4(ra), u1[s] = ld_cluster_f4(ra + 16);
-                        }
-                    }
-                    v0 = u0[0], v1 = u1[0];
-#pragma unroll
-                    for (int s = 1; s < G::MAX_S; ++s) {
-                        if (s < S) {
-                            v0.x += u0[s].x, v0.y += u0[s].y, v0.z += u0[s].z, v0.w += u0[s].w;
-                            v1.x += u1[s].x, v1.y += u1[s].y, v1.z += u1[s].z, v1.w += u1[s].w;
+                    for (int sp_ = 0; sp_ < G::MAX_S; ++sp_) {
+                        if (sp_ < S) {
+                            const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)sp_);
+                            u0[i][sp_] = ld_cluster_f4(ra), u1[i][sp_] = ld_cluster_f4(ra + 16);
                         }
                     }
                 }
+            }
+#pragma unroll
+            for (int i = 0; i < G::MAX_ITEMS; ++i) {
+                if (mm[i] < 0) continue;
+                float4 v0 = u0[i][0], v1 = u1[i][0];
+#pragma unroll
+                for (int sp_ = 1; sp_ < G::MAX_S; ++sp_) {
+                    if (sp_ < S) {
+                        v0.x += u0[i][sp_].x, v0.y += u0[i][sp_].y, v0.z += u0[i][sp_].z, v0.w += u0[i][sp_].w;
+                        v1.x += u1[i][sp_].x, v1.y += u1[i][sp_].y, v1.z += u1[i][sp_].z, v1.w += u1[i][sp_].w;
+                    }
+                }
                 float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                epi.apply(m, n, a, side[i]);
+                epi.apply(mm[i], nn[i], a, side[i]);
             }
         }
     }
