@@ -19,11 +19,10 @@
 // groups.  Group g takes the key blocks b with b % 2 == g and keeps its own
 // (max, sum, O) state, S accumulator and P tile, so that one group's
 // exponentials overlap the other's tensor-memory traffic and UMMAs.
-// A key range longer than CH blocks is split over several CTAs; every group of
-// every split writes its unnormalised (O, m, l) state, and the CTA that finishes
-// last (a counter per query tile) merges all states in (split, group) order and
-// writes the output.  With a single split the two groups are merged in shared
-// memory instead.
+// At the end the two groups' states are merged in shared memory.  A key range
+// longer than CH blocks is split over several CTAs; each writes its unnormalised
+// (O, m, l) state, and the CTA that finishes last (a counter per query tile)
+// merges the states in split order and writes the output.
 // CH depends only on the configuration, so a frame's result does not depend on
 // which other frames share its pass.
 #pragma once
@@ -306,45 +305,58 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         }
         const int row = qt * 128 + trow;
         const size_t item_q = (size_t)z * pl.QT + qt;      // (frame, head, query tile)
-        if (nsplit == 1) {
-            // ---- one CTA holds the whole window: group 1 parks its state, group 0 folds it in ----
-            named_bar_sync(1, 256);                        // both groups are past their last UMMA: the P tiles are free
-            if (g == 1) {
-                float4 *po = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);
+        // ---- the two groups of this CTA first: group 1 parks its state, group 0 folds it in ----
+        named_bar_sync(1, 256);                            // both groups are past their last UMMA: the P tiles are free
+        if (g == 1) {
+            float4 *po = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);
 #pragma unroll
-                for (int e = 0; e < 64; e += 4) po[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
-                parkML[trow] = make_float2(m_run, l_run);
+            for (int e = 0; e < 64; e += 4) po[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
+            parkML[trow] = make_float2(m_run, l_run);
+        }
+        named_bar_sync(1, 256);
+        float m_cta = m_run, l_cta = l_run;
+        if (g == 0) {
+            const float2 ml1 = parkML[trow];
+            m_cta = fmaxf(m_run, ml1.x);
+            const float w0 = ex2_approx(m_run - m_cta), w1 = ex2_approx(ml1.x - m_cta);
+            l_cta = l_run * w0 + ml1.y * w1;
+            const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)trow * A::OROW);
+#pragma unroll
+            for (int e = 0; e < 64; e += 4) {
+                const float4 v = po[e >> 2];
+                O[e] = fmaf(O[e], w0, v.x * w1), O[e + 1] = fmaf(O[e + 1], w0, v.y * w1);
+                O[e + 2] = fmaf(O[e + 2], w0, v.z * w1), O[e + 3] = fmaf(O[e + 3], w0, v.w * w1);
             }
-            named_bar_sync(1, 256);
+        }
+        if (nsplit == 1) {
             if (g == 0 && row < D.T) {
-                const float2 ml1 = parkML[trow];
-                const float m = fmaxf(m_run, ml1.x);
-                const float w0 = ex2_approx(m_run - m), w1 = ex2_approx(ml1.x - m);
-                const float inv = 1.0f / (l_run * w0 + ml1.y * w1);
-                const float a0 = w0 * inv, a1 = w1 * inv;
-                const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)trow * A::OROW);
+                const float inv = 1.0f / l_cta;
                 bf16 *o = out + (size_t)(j * D.T + row) * D.d + h * 64;
 #pragma unroll
                 for (int e = 0; e < 64; e += 8) {
-                    const float4 v0 = po[e >> 2], v1 = po[(e >> 2) + 1];
-                    float t[8] = {fmaf(O[e], a0, v0.x * a1),     fmaf(O[e + 1], a0, v0.y * a1),
-                                  fmaf(O[e + 2], a0, v0.z * a1), fmaf(O[e + 3], a0, v0.w * a1),
-                                  fmaf(O[e + 4], a0, v1.x * a1), fmaf(O[e + 5], a0, v1.y * a1),
-                                  fmaf(O[e + 6], a0, v1.z * a1), fmaf(O[e + 7], a0, v1.w * a1)};
+                    float t[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) t[u] = O[e + u] * inv;
                     *reinterpret_cast<uint4 *>(o + e) = pack_bf16x8(t);
                 }
             }
         } else {
-            // ---- both groups publish their state; the CTA that finishes last merges all 2*nsplit states ----
-            const size_t st0 = item_q * (2 * pl.MAXSPLIT) * 128;                     // first state row of this query tile
-            {
-                const size_t item = st0 + (size_t)(2 * split + g) * 128 + trow;
+            // ---- publish this CTA's state; the CTA that finishes last merges the splits in split order ----
+            const size_t st0 = item_q * pl.MAXSPLIT * 128;                           // first state row of this query tile
+            if (g == 0) {
+                const size_t item = st0 + (size_t)split * 128 + trow;
                 float4 *po4 = reinterpret_cast<float4 *>(part_o + item * 64);
+                float4 *ps4 = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);     // own copy for the merge
 #pragma unroll
-                for (int e = 0; e < 64; e += 4) po4[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
-                part_ml[item] = make_float2(m_run, l_run);
+                for (int e = 0; e < 64; e += 4) {
+                    const float4 v = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
+                    po4[e >> 2] = v;
+                    ps4[e >> 2] = v;
+                }
+                part_ml[item] = make_float2(m_cta, l_cta);
+                parkML[trow] = make_float2(m_cta, l_cta);
+                __threadfence();
             }
-            __threadfence();
             named_bar_sync(1, 256);
             if (threadIdx.x == 64) {
                 const unsigned int prev = atomicAdd(counters + item_q, 1u);
@@ -355,37 +367,43 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             named_bar_sync(1, 256);
             if (*last_flag) {
                 __threadfence();
-                const int ns = 2 * nsplit;                 // states, in (split, group) order
                 for (int it = (int)threadIdx.x - 64; it < 128 * 8; it += 256) {
                     const int r = it >> 3, ch = it & 7;
                     const int orow = qt * 128 + r;
                     if (orow >= D.T) continue;
                     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                     float l = 0.f, mx = -INFINITY;
-                    for (int s0 = 0; s0 < ns; s0 += 6) {
-                        // six states at a time, all loads in flight together
-                        float2 ml[6];
-                        float4 v0[6], v1[6];
+                    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+                        // four splits at a time, all loads in flight together; this CTA's own state comes from
+                        // shared memory (same values as its published copy)
+                        float2 ml[4];
+                        float4 v0[4], v1[4];
 #pragma unroll
-                        for (int u = 0; u < 6; ++u) {
-                            const int s = s0 + u < ns ? s0 + u : ns - 1;
-                            const size_t item = st0 + (size_t)s * 128 + r;
-                            ml[u] = __ldcg(&part_ml[item]);
-                            const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch * 8);
-                            v0[u] = __ldcg(po), v1[u] = __ldcg(po + 1);
+                        for (int u = 0; u < 4; ++u) {
+                            const int s = s0 + u < nsplit ? s0 + u : nsplit - 1;
+                            if (s == split) {
+                                ml[u] = parkML[r];
+                                const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)r * A::OROW + ch * 8);
+                                v0[u] = po[0], v1[u] = po[1];
+                            } else {
+                                const size_t item = st0 + (size_t)s * 128 + r;
+                                ml[u] = __ldcg(&part_ml[item]);
+                                const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch * 8);
+                                v0[u] = __ldcg(po), v1[u] = __ldcg(po + 1);
+                            }
                         }
                         float mb = mx;
 #pragma unroll
-                        for (int u = 0; u < 6; ++u)
-                            if (s0 + u < ns) mb = fmaxf(mb, ml[u].x);
+                        for (int u = 0; u < 4; ++u)
+                            if (s0 + u < nsplit) mb = fmaxf(mb, ml[u].x);
                         const float fo = ex2_approx(mx - mb);          // rescale of what was merged so far (0 at first)
                         l *= fo;
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc[e] *= fo;
                         mx = mb;
 #pragma unroll
-                        for (int u = 0; u < 6; ++u) {
-                            if (s0 + u < ns) {
+                        for (int u = 0; u < 4; ++u) {
+                            if (s0 + u < nsplit) {
                                 const float w = ex2_approx(ml[u].x - mx);
                                 l = fmaf(ml[u].y, w, l);
                                 acc[0] = fmaf(v0[u].x, w, acc[0]), acc[1] = fmaf(v0[u].y, w, acc[1]);

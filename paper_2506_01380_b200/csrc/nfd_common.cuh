@@ -74,6 +74,11 @@ struct RopeTab {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Pull a byte range towards L2 (addr 16-byte aligned, bytes a multiple of 16).
+__device__ __forceinline__ void bulk_prefetch_l2(const void *addr, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(addr), "r"(bytes) : "memory");
+}
+
 // ---- timeline instrumentation (compiled out unless NFD_TRACE is defined) ------
 // With -DNFD_TRACE every CTA of the instrumented kernels appends one record
 // (kernel kind, SM, start and end on the global nanosecond timer) to a buffer

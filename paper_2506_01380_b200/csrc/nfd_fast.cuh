@@ -24,7 +24,7 @@ struct FastState {
     int n_sm = 148;
     size_t a_rows = 0;     // rows of every activation buffer (NFD_MAX_PASS_FRAMES * T)
     AttnPlan plan;         // KB == 0: tensor-core attention not available for this shape
-    float *part_o = nullptr;           // per (split, softmax group) states of the attention kernel
+    float *part_o = nullptr;           // per-split states of the attention kernel
     float2 *part_ml = nullptr;
     unsigned int *attn_counters = nullptr;   // one per (frame, head, query tile); zero between launches
     size_t cache_rows = 0;
@@ -65,7 +65,7 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
         pl.MAXSPLIT = ((D.W + 1) * pl.BPF + pl.CH - 1) / pl.CH;
         if (pl.MAXSPLIT > 1) {
             const size_t tiles = (size_t)NFD_MAX_PASS_FRAMES * D.H * pl.QT;
-            const size_t items = tiles * 2 * pl.MAXSPLIT * 128;      // one state per (split, softmax group)
+            const size_t items = tiles * pl.MAXSPLIT * 128;          // one state per split
             if (cudaMalloc((void **)&fs.part_o, items * 64 * sizeof(float)) != cudaSuccess ||
                 cudaMalloc((void **)&fs.part_ml, items * sizeof(float2)) != cudaSuccess ||
                 cudaMalloc((void **)&fs.attn_counters, tiles * sizeof(unsigned int)) != cudaSuccess ||

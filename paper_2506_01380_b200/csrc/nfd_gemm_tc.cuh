@@ -121,13 +121,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tma_load_2d(smem_u32(sA + s * G::A_BYTES), &tmA, full0 + 8 * s, (kb0 + kb) * 64, m0);
                 tma_load_2d(smem_u32(sB + s * G::B_BYTES), &tmB, full0 + 8 * s, (kb0 + kb) * 64, n0);
             }
-        } else if (lane == 1 && pf.bytes) {
-            // this CTA's slice of the next GEMM's weights, towards L2 in 8 KiB pieces
+        } else if (lane == 1) {
+            // this CTA's slice of the next GEMM's weights, towards L2 in 8 KiB pieces, and whatever the
+            // epilogue functor knows the next kernel will read
             const unsigned long long n_cta = (unsigned long long)gridDim.x * gridDim.y;
             const unsigned long long cta = (unsigned long long)blockIdx.y * gridDim.x + blockIdx.x;
+            epi.prefetch((unsigned int)cta, (unsigned int)n_cta);
             const unsigned long long per = ((pf.bytes / n_cta + 15) / 16 + 1) * 16;
             unsigned long long b = cta * per, e = b + per;
             if (e > pf.bytes) e = pf.bytes;
+            if (!pf.bytes) b = e = 0;
             for (; b < e; b += 8192) {
                 const unsigned long long n = e - b < 8192 ? e - b : 8192;
                 bulk_prefetch_l2(reinterpret_cast<const uint8_t *>(pf.ptr) + b, (uint32_t)n);

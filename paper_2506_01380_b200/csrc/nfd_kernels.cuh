@@ -346,6 +346,22 @@ template <typename TS> struct EpiQKV {
     int layer;
     const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by the tensor-core path
     int n_rows;                 // nf*T: rows of the pass (q is [H][n_rows][dh])
+    // Pull the cached K/V pages that the attention kernel of this layer is about to read towards L2 (the
+    // pages of frames before this pass are final); each CTA of the launch takes a slice of every page.
+    __device__ __forceinline__ void prefetch(unsigned int cta, unsigned int n_cta) const {
+        if (sizeof(TS) != 2) return;
+        const FrameDesc fr = sp->fr[0];
+        const size_t page_bytes = D.page_elems * sizeof(TS);
+        const size_t per = ((page_bytes / n_cta + 15) / 16) * 16;
+        const size_t b = (size_t)cta * per;
+        if (b >= page_bytes) return;
+        const unsigned int n = (unsigned int)(page_bytes - b < per ? page_bytes - b : per);
+        for (int g = fr.win_first; g < fr.first_new; ++g) {
+            const size_t off = kv_page_offset(D, fr.stream, layer, g);
+            bulk_prefetch_l2(reinterpret_cast<const unsigned char *>(kc + off) + b, n);
+            bulk_prefetch_l2(reinterpret_cast<const unsigned char *>(vc + off) + b, n);
+        }
+    }
     struct Side {
         uint4 bias;
         float4 c01, c23;        // (cos, sin) of four adjacent pairs
@@ -425,6 +441,7 @@ template <typename TS> struct EpiGateRes {
     const float *gate;      // mod + layer offset + chunk offset
     size_t row_stride;
     Dims D;
+    __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     struct Side {
         uint4 bias;
         float4 g0, g1, z0, z1;
@@ -467,6 +484,7 @@ template <typename TS> struct EpiGelu {
     const TS *bias;
     TS *out;
     int N;
+    __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     struct Side {
         uint4 bias;
     };
@@ -493,6 +511,7 @@ template <typename TS> struct EpiFinal {
     const StepParams *sp;
     const TS *bias;
     Dims D;
+    __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     struct Side {
         int unused;
     };
