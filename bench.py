@@ -122,6 +122,18 @@ def class_work(cfg, T, n_ctx):
     }
 
 
+# DRAM bytes (read + write) of one launch from the ncu captures summarised under profiles/ (same kernels,
+# 2-layer slice of this shape; one launch of a kernel moves the same bytes whatever the layer count).
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "attention": 24.13e6,               # profiles/ncu_attention_nfd310m_k1.txt
+    "gemm_qkv_rope_kvstore": 31.33e6,   # profiles/ncu_gemm_nfd310m_k1.txt (includes the K/V page prefetch for attention)
+    "gemm_out_gate_res": 12.68e6,
+    "gemm_fc1_gelu": 17.60e6,
+    "gemm_fc2_gate_res": 19.24e6,
+    "adaln_norm": 5.54e6,
+}
+
+
 def roofline_of(cfg, T, n_ctx, prof, pk):
     work = class_work(cfg, T, n_ctx)
     total = sum(ms for _, ms in prof.values()) or 1.0
@@ -145,7 +157,9 @@ def roofline_of(cfg, T, n_ctx, prof, pk):
         ach, peak, unit, bound = w["bytes"] / dur / 1e9, pk["hbm"], "GB/s", "hbm"
     return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
             "frac": round(ach / peak, 4), "peak_source": pk["src"] + (" (sustained)" if bound == "tensor" else ""),
-            "avg_launch_us": round(dur * 1e6, 2), "share_of_step": shares.get(name), "traffic": None}, shares
+            "avg_launch_us": round(dur * 1e6, 2), "share_of_step": shares.get(name),
+            "algorithmic_bytes": w["bytes"], "algorithmic_flops": w["flops"],
+            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name)}, shares
 
 
 # ---------------------------------------------------------------------------
