@@ -41,7 +41,6 @@ template <int BN> struct GemmCfg {
     static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
-    static constexpr int MAX_ITEMS = 2;                        // epilogue items in flight together per thread
     static constexpr int MAX_S = 4;                            // largest cluster split
     static constexpr int MIN_CTAS = 1;
     static_assert(STAGE_BYTES <= RING_BYTES, "staging tile must fit the operand ring");
@@ -58,6 +57,7 @@ __global__ void __launch_bounds__(GemmCfg<BN>::THREADS, GemmCfg<BN>::MIN_CTAS)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int K,
           int S, Epi epi, L2Prefetch pf, int *status) {
     using G = GemmCfg<BN>;
+    constexpr int MAX_ITEMS = Epi::kBatch;                   // epilogue items in flight together per thread
     extern __shared__ uint8_t smem_raw[];
     NFD_TRACE_T0();
     // blockIdx.x = n_tile * S + split; the S splits of a tile form one cluster
@@ -100,7 +100,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const int et = (int)threadIdx.x - 64;                    // 0..255 for the epilogue warps
     const int n_items = rows_per * CPR;                      // items of this CTA's row slice
     const int r_base = (S > 1 ? (int)cluster_ctarank() : 0) * rows_per;   // first tile row of the slice
-    typename Epi::Side side[G::MAX_ITEMS];
+    typename Epi::Side side[MAX_ITEMS];
 
     if (warp == 0) {
         if (lane == 0) {
@@ -159,7 +159,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         pdl_wait();
         // side inputs of the first items (bias, gate, residual, rotary table), fetched while the UMMAs run
 #pragma unroll
-        for (int i = 0; i < G::MAX_ITEMS; ++i) {
+        for (int i = 0; i < MAX_ITEMS; ++i) {
             const int it = et + i * G::EPI_THREADS;
             if (it < n_items) {
                 const int m = m0 + r_base + it / CPR, n = n0 + (it % CPR) * 8;
@@ -194,50 +194,58 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __syncthreads();
     NFD_TRACE_MARK_T(TRK_OTHER + 3, 64);
     if (warp >= 2) {
-        // Items in batches of MAX_ITEMS.  Phase A issues every load of the batch (side inputs, and the S
-        // partials, remote ones through distributed shared memory: their latency is long); phase B sums the
-        // partials in split order and runs the fused epilogue, 8 adjacent columns per item.
+        // Items in batches of MAX_ITEMS: first every side input of the batch is requested, then the items are
+        // finished two at a time: all loads of the S partials of the pair (remote ones come through distributed
+        // shared memory and take long), the sum in split order, the fused epilogue (8 adjacent columns per item).
         const uint32_t stage_u32 = smem_u32(stage);
-        for (int i0 = 0; i0 * G::EPI_THREADS < n_items; i0 += G::MAX_ITEMS) {
-            float4 u0[G::MAX_ITEMS][G::MAX_S], u1[G::MAX_ITEMS][G::MAX_S];
-            int mm[G::MAX_ITEMS], nn[G::MAX_ITEMS];
+        for (int i0 = 0; i0 * G::EPI_THREADS < n_items; i0 += MAX_ITEMS) {
+            int mm[MAX_ITEMS], nn[MAX_ITEMS], tr[MAX_ITEMS];
 #pragma unroll
-            for (int i = 0; i < G::MAX_ITEMS; ++i) {
+            for (int i = 0; i < MAX_ITEMS; ++i) {
                 const int it = et + (i0 + i) * G::EPI_THREADS;
-                const int trow = r_base + it / CPR, cc = it % CPR;
-                mm[i] = m0 + trow, nn[i] = n0 + cc * 8;
-                if (it >= n_items || mm[i] >= M || nn[i] >= N) {
+                tr[i] = r_base + it / CPR;
+                mm[i] = m0 + tr[i], nn[i] = n0 + (it % CPR) * 8;
+                if (it >= n_items || mm[i] >= M || nn[i] >= N)
                     mm[i] = -1;
-                    continue;
-                }
-                if (i0 > 0) epi.load(mm[i], nn[i], side[i]);
-                const uint32_t off = (uint32_t)(trow * G::SROW + cc * 8) * 4;
-                if (S == 1) {
-                    const float *p = stage + (size_t)trow * G::SROW + cc * 8;
-                    u0[i][0] = *reinterpret_cast<const float4 *>(p), u1[i][0] = *reinterpret_cast<const float4 *>(p + 4);
-                } else {
+                else if (i0 > 0)
+                    epi.load(mm[i], nn[i], side[i]);
+            }
 #pragma unroll
-                    for (int sp_ = 0; sp_ < G::MAX_S; ++sp_) {
-                        if (sp_ < S) {
-                            const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)sp_);
-                            u0[i][sp_] = ld_cluster_f4(ra), u1[i][sp_] = ld_cluster_f4(ra + 16);
+            for (int j0 = 0; j0 < MAX_ITEMS; j0 += 2) {
+                float4 u0[2][G::MAX_S], u1[2][G::MAX_S];
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int i = j0 + jj;
+                    if (i >= MAX_ITEMS || mm[i] < 0) continue;
+                    const uint32_t off = (uint32_t)(tr[i] * G::SROW + (nn[i] - n0)) * 4;
+                    if (S == 1) {
+                        const float *p = stage + (size_t)tr[i] * G::SROW + (nn[i] - n0);
+                        u0[jj][0] = *reinterpret_cast<const float4 *>(p), u1[jj][0] = *reinterpret_cast<const float4 *>(p + 4);
+                    } else {
+#pragma unroll
+                        for (int sp_ = 0; sp_ < G::MAX_S; ++sp_) {
+                            if (sp_ < S) {
+                                const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)sp_);
+                                u0[jj][sp_] = ld_cluster_f4(ra), u1[jj][sp_] = ld_cluster_f4(ra + 16);
+                            }
                         }
                     }
                 }
-            }
 #pragma unroll
-            for (int i = 0; i < G::MAX_ITEMS; ++i) {
-                if (mm[i] < 0) continue;
-                float4 v0 = u0[i][0], v1 = u1[i][0];
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int i = j0 + jj;
+                    if (i >= MAX_ITEMS || mm[i] < 0) continue;
+                    float4 v0 = u0[jj][0], v1 = u1[jj][0];
 #pragma unroll
-                for (int sp_ = 1; sp_ < G::MAX_S; ++sp_) {
-                    if (sp_ < S) {
-                        v0.x += u0[i][sp_].x, v0.y += u0[i][sp_].y, v0.z += u0[i][sp_].z, v0.w += u0[i][sp_].w;
-                        v1.x += u1[i][sp_].x, v1.y += u1[i][sp_].y, v1.z += u1[i][sp_].z, v1.w += u1[i][sp_].w;
+                    for (int sp_ = 1; sp_ < G::MAX_S; ++sp_) {
+                        if (sp_ < S) {
+                            v0.x += u0[jj][sp_].x, v0.y += u0[jj][sp_].y, v0.z += u0[jj][sp_].z, v0.w += u0[jj][sp_].w;
+                            v1.x += u1[jj][sp_].x, v1.y += u1[jj][sp_].y, v1.z += u1[jj][sp_].z, v1.w += u1[jj][sp_].w;
+                        }
                     }
+                    float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                    epi.apply(mm[i], nn[i], a, side[i]);
                 }
-                float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                epi.apply(mm[i], nn[i], a, side[i]);
             }
         }
     }

@@ -362,10 +362,11 @@ template <typename TS> struct EpiQKV {
             bulk_prefetch_l2(reinterpret_cast<const unsigned char *>(vc + off) + b, n);
         }
     }
+    static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
     struct Side {
         uint4 bias;
         float4 c01, c23;        // (cos, sin) of four adjacent pairs
-        FrameDesc fr;
+        int stream, frame;      // of the token's frame
     };
     __device__ __forceinline__ void load(int m, int n, Side &s) const {
         s.bias = *reinterpret_cast<const uint4 *>(bias + n);
@@ -375,7 +376,8 @@ template <typename TS> struct EpiQKV {
             const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
             s.c01 = cs[0], s.c23 = cs[1];
         }
-        s.fr = sp->fr[m / D.T];
+        const FrameDesc &f = sp->fr[m / D.T];
+        s.stream = f.stream, s.frame = f.frame;
     }
     __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
         float b[8];
@@ -399,7 +401,7 @@ template <typename TS> struct EpiQKV {
         if (which == 0) {
             dst = q + ((size_t)head * ((size_t)n_rows) + m) * D.dh + e;
         } else {
-            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, s.fr.stream, layer, s.fr.frame) +
+            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, s.stream, layer, s.frame) +
                   ((size_t)head * D.T + tok) * D.dh + e;
         }
         *reinterpret_cast<uint4 *>(dst) = pack_bf16x8(a);
@@ -442,6 +444,7 @@ template <typename TS> struct EpiGateRes {
     size_t row_stride;
     Dims D;
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
+    static constexpr int kBatch = 2;        // epilogue items a thread keeps in flight together
     struct Side {
         uint4 bias;
         float4 g0, g1, z0, z1;
@@ -485,6 +488,7 @@ template <typename TS> struct EpiGelu {
     TS *out;
     int N;
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
+    static constexpr int kBatch = 8;        // epilogue items a thread keeps in flight together
     struct Side {
         uint4 bias;
     };
@@ -512,6 +516,7 @@ template <typename TS> struct EpiFinal {
     const TS *bias;
     Dims D;
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
+    static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
     struct Side {
         int unused;
     };
