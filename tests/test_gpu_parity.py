@@ -344,3 +344,31 @@ def test_deferred_commit_equals_immediate_commit(name):
         Kb, Vb = eager.kv_read(L - 1, f)
         assert torch.equal(Ka, Kb) and torch.equal(Va, Vb)
     assert lazy.status() == 0 and eager.status() == 0
+
+
+def test_batch8_streams_at_model_width_match_single_streams():
+    """Config 5's structure (8 independent streams, 32-frame context) on a 2-layer slice of the 310M-class
+    width: one batched speculation must give bitwise the frames and caches of eight single-stream ones."""
+    from paper_2506_01380_b200.nfd import NFD
+    torch = _torch()
+    cfg = I.make_cfg("nfd310m_b8", n_layers=2)
+    w = I.make_weights(cfg, 9, "stress")
+    gb, gs = NFD(cfg, w), NFD(cfg, w)
+    S, k, n = cfg["n_steps"], 1, 8
+    for s in range(n):
+        x0 = dev(I.round_bf16(I.make_latents(cfg, 2, 300 + s)))
+        acts = I.make_actions_uniform(cfg, 2, 400 + s)
+        gb.commit_frame(x0, acts, None, stream=s)
+        gs.commit_frame(x0, acts, None, stream=s)
+    noise = dev(I.round_bf16(np.stack([I.make_noise(cfg, S, k, 500 + s) for s in range(n)], axis=1)))   # [S,n,k,...]
+    actions = [(3 * s + 1) % cfg["n_actions"] for s in range(n)]
+    xb = gb.speculate_batched(list(range(n)), k, actions, noise)
+    for s in range(n):
+        xs = gs.speculate(k, actions[s], noise[:, s].contiguous(), stream=s)
+        assert torch.equal(xs, xb[s]), f"stream {s}"
+    for s in range(n):
+        gb.rollback(1, stream=s)
+        gs.rollback(1, stream=s)
+        assert gb.kv_state(s) == gs.kv_state(s) == (3, 0, 0)
+        assert gb.kv_hash(s) == gs.kv_hash(s)
+    assert gb.status() == 0 and gs.status() == 0
