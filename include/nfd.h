@@ -86,7 +86,7 @@ typedef struct {
 
 /* Create a context.  `cuda_stream` is a cudaStream_t (NULL = legacy default
  * stream).  Validates cfg (NFD_E_BADCFG), copies/repacks the weights, allocates
- * the cache: n_streams x n_layers x (W + k_max) frame pages of K and of V.
+ * the cache: n_streams x n_layers x (W + 2 k_max) frame pages of K and of V.
  * Synchronises the stream before returning. */
 int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cuda_stream);
 int nfd_destroy(nfd_ctx *ctx);
@@ -130,7 +130,16 @@ int nfd_commit_frame(nfd_ctx *ctx, int stream, const float *x0, int n, const int
  * over the k frames decoded together, then append the k clean frames as
  * TENTATIVE.  noise dev fp32 [S,k,C,H,W] (N(0,1): step 0 is the initial sample,
  * step s>0 the re-noising draw); ctx_noise dev [k,C,H,W] or NULL; x0_out dev
- * fp32 [k,C,H,W] receives the clean frames.  Requires no tentative frames. */
+ * fp32 [k,C,H,W] receives the clean frames.  Requires no tentative frames.
+ *
+ * The K/V pages of the k frames are not written by this call: the library keeps
+ * a copy of the clean frames, their context noise and the action, counts the
+ * frames as tentative, and lets them ride along (K/V only) in the first
+ * denoising pass of the next nfd_speculate on this batch slot -- the paper's
+ * "compute and cache their KVs during the first denoising step" (Appendix,
+ * KV caching).  Any call that needs the pages earlier (nfd_kv_hash,
+ * nfd_kv_read, nfd_denoise_step*, nfd_commit_frame) writes them first.  Results
+ * are bitwise those of committing at once (option "lazy_commit" = 0). */
 int nfd_speculate(nfd_ctx *ctx, int stream, int k, int action, const float *noise, const float *ctx_noise,
                   float *x0_out);
 
@@ -141,8 +150,9 @@ int nfd_speculate_batched(nfd_ctx *ctx, int n, const int *streams, int k, const 
 
 /* Resolve a speculation (Section 4.2: frames after the first action mismatch are
  * discarded, generation resumes from the last verified frame): the first
- * n_accept tentative frames become committed, the rest are dropped.  Counters
- * only; no data moves.  0 <= n_accept <= n_tentative. */
+ * n_accept tentative frames become committed, the rest are dropped (frames whose
+ * commit was still deferred are simply forgotten).  Counters only; no data
+ * moves.  0 <= n_accept <= n_tentative. */
 int nfd_rollback(nfd_ctx *ctx, int stream, int n_accept);
 
 /* Cache counters (host ints, any may be NULL): committed frames, tentative
@@ -166,7 +176,7 @@ int nfd_kv_read(nfd_ctx *ctx, int stream, int layer, int frame, float *k_out, fl
  * storage type, [n_q_frames*T, n_heads*head_dim].  The data are first copied
  * into cache pages of batch slot 0 (which is reset), then the same attention
  * kernel the forward pass uses runs on them.
- * n_kv_frames <= W + k_max, n_q_frames <= k_max, window <= W. */
+ * n_kv_frames <= W + 2 k_max, n_q_frames <= k_max, window <= W. */
 int nfd_attention(nfd_ctx *ctx, const void *q, const void *k, const void *v, int n_q_frames, int n_kv_frames,
                   int window, void *out);
 
@@ -231,7 +241,9 @@ const char *nfd_profile_class_name(int id);
 
 /* Run-time switches, for tests and profiling: "graph" 0/1 (replay CUDA graphs
  * or launch kernels directly), "fast" 0/1 (tensor-core kernels or the plain
- * validation kernels; bf16 only).  Returns NFD_E_RANGE for unknown names. */
+ * validation kernels; bf16 only), "lazy_commit" 0/1 (defer the commit of
+ * speculated frames into the next speculation's first pass, or commit them at
+ * once).  Returns NFD_E_RANGE for unknown names. */
 int nfd_set_option(nfd_ctx *ctx, const char *name, int value);
 
 const char *nfd_strerror(int code);
