@@ -243,7 +243,11 @@ const char *nfd_profile_class_name(int id);
  * or launch kernels directly), "fast" 0/1 (tensor-core kernels or the plain
  * validation kernels; bf16 only), "lazy_commit" 0/1 (defer the commit of
  * speculated frames into the next speculation's first pass, or commit them at
- * once).  Returns NFD_E_RANGE for unknown names. */
+ * once), "fuse_ln" 0/1 (bf16 tensor-core path: fold the two adaLN LayerNorms of
+ * every block into the epilogues of the neighbouring GEMMs, or run them as
+ * kernels of their own; the two differ by bf16 rounding of the GEMM operand
+ * only).  Changing "fast" or "fuse_ln" empties the modulation cache.  Returns
+ * NFD_E_RANGE for unknown names. */
 int nfd_set_option(nfd_ctx *ctx, const char *name, int value);
 
 const char *nfd_strerror(int code);

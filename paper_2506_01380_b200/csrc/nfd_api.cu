@@ -53,6 +53,7 @@ struct nfd_ctx {
     std::vector<void *> w_mod, b_mod, w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2;
     // device arrays of pointers for the GEMV kernels
     void **dp_wmod = nullptr, **dp_bmod = nullptr, **dp_t1 = nullptr, **dp_t2 = nullptr, **dp_fmod = nullptr;
+    void **dp_wqkv = nullptr, **dp_bqkv = nullptr, **dp_wfc1 = nullptr, **dp_bfc1 = nullptr;
     RopeTab *d_rope = nullptr;
 
     void *kc = nullptr, *vc = nullptr;          // [n_streams][L][R][H][T][dh]
@@ -83,6 +84,18 @@ struct nfd_ctx {
         long long last_use = -1;
     };
     std::vector<CondSlot> cond_slots;
+    // Folded LayerNorm (tensor-core path): the in-layer adaLN kernels are replaced by work in the epilogues
+    // of the neighbouring GEMMs.  uvtab holds, per cache slot and layer, the (u, v) pairs of the QKV and
+    // first MLP projections; ln_stats the row-sum partials of z.
+    bool fuse_ln = true;
+    float2 *uvtab = nullptr;                    // [n_slots][L][3d + dm]
+    float2 *ln_stats = nullptr;                 // [Nq_max][d / 32]
+    bool fold_active() const {
+        const int d = D.d, dm = D.dm;
+        // (a 128-row GEMM tile must not span more frames than the kernel keeps (u, v) rows for)
+        return fuse_ln && fast && bf16_mode && fs.ready && d % 32 == 0 && d >= 64 && dm % 8 == 0 && dm >= 64 &&
+               127 / D.T + 2 <= LnFold::kMaxFrames;
+    }
     long long pass_no = 0, cond_hits = 0, cond_misses = 0;
     std::map<int, GraphEntry> graphs;
 
@@ -195,7 +208,7 @@ static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
 // ---------------------------------------------------------------------------
 // One forward pass, enqueued on the context's stream.
 // ---------------------------------------------------------------------------
-#define NFD_COND_SLOTS 96       // rows of the modulation cache (> NFD_MAX_PASS_FRAMES)
+#define NFD_COND_SLOTS 256      // rows of the modulation cache (> NFD_MAX_PASS_FRAMES)
 
 enum { CLS_PARAMS = 0, CLS_COND, CLS_PATCH, CLS_ADALN, CLS_GEMM_QKV, CLS_ATTN, CLS_GEMM_O, CLS_GEMM_FC1,
        CLS_GEMM_FC2, CLS_HEAD, CLS_SAMPLER, CLS_CACHE, CLS_COUNT };
@@ -245,13 +258,19 @@ static void prof_mark(nfd_ctx *c, bool stop) {
 
 template <typename TS, typename Epi>
 static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind,
-                        const void *next_w = nullptr, size_t next_elems = 0) {
+                        const void *next_w = nullptr, size_t next_elems = 0, bool folded = false) {
     prof_mark(c, false);
     // the next GEMM's weights, pulled towards L2 by this launch
     const L2Prefetch pf{next_w, next_w ? (unsigned long long)(next_elems * sizeof(TS)) & ~15ull : 0ull};
     if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, A, Wt, M, N, K, epi, tc_kind, pf)) {
         prof_mark(c, true);
         c->launches++;
+        return;
+    }
+    if (folded) {
+        // the plain kernel knows nothing of the folded LayerNorm: fail the pass rather than compute garbage
+        fprintf(stderr, "libnfd: tensor-core GEMM unavailable for a pass with folded LayerNorm\n");
+        if (!c->launch_err) c->launch_err = cudaErrorNotSupported;
         return;
     }
     dim3 grid((N + 63) / 64, (M + 63) / 64);
@@ -288,6 +307,8 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     const int d = D.d, L = D.L, M = nf * D.T;
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
+    const size_t uv_row = (size_t)L * (3 * d + D.dm);
+    const bool fold = c->fold_active();
     // conditioning: only for the (t, action) pairs that are not in the modulation cache
     c->cls = CLS_COND;
     if (c->h_sp.nc > 0) {
@@ -304,41 +325,59 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
         PLAUNCH(c, (k_gemv<TS, GEMV_MOD>), dim3((2 * d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_fmod,
                 (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, (const float *)c->sc, c->fmod, d, 2 * d,
                 (size_t)2 * d, (size_t)0);
+        if (fold)
+            PLAUNCH(c, (k_modw<TS>), dim3((3 * d + D.dm + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wqkv,
+                    (const TS *const *)c->dp_bqkv, (const TS *const *)c->dp_wfc1, (const TS *const *)c->dp_bfc1,
+                    (const float *)c->mod, mod_row, c->uvtab, uv_row, d, D.dm);
     }
     // tokens
     c->cls = CLS_PATCH;
     if (c->bf16_mode && c->fast)
         PLAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, (const RopeTab *)c->d_rope, c->rope_cs);
     PLAUNCH(c, (k_patch_embed<TS>), dim3((M + PE_TOK - 1) / PE_TOK, (d + 255) / 256), 256, PE_TOK * D.P * sizeof(float), sp, D,
-            (const TS *)c->w_pe_io, (const TS *)c->b_pe, c->z);
+            (const TS *)c->w_pe_io, (const TS *)c->b_pe, c->z, fold ? (TS *)c->hbuf : (TS *)nullptr, c->ln_stats,
+            (const float *)c->mod + d, mod_row);
     const int ln_grid = (M + 3) / 4;
     for (int l = 0; l < L; ++l) {
         const float *modl = c->mod + (size_t)l * 6 * d;
-        c->cls = CLS_ADALN;
-        PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row, (size_t)0,
-                (size_t)d);
+        // with the folded LayerNorm hbuf already holds z*(1+scale) and ln_stats the row sums of z
+        LnFold lq{nullptr, uv_row, c->ln_stats, d / 32, D.norm, D.eps, sp, D.T}, lm = lq;
+        if (fold) {
+            lq.uv = c->uvtab + (size_t)l * (3 * d + D.dm);
+            lm.uv = lq.uv + 3 * d;
+        } else {
+            c->cls = CLS_ADALN;
+            PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row,
+                    (size_t)0, (size_t)d);
+        }
         EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l,
-                      c->rope_cs, M};
+                      c->rope_cs, M, lq};
         c->cls = CLS_GEMM_QKV;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV, c->w_o[l],
-                        (size_t)d * d);
+                        (size_t)d * d, fold);
         if (kind == 1 && l == L - 1) break;      // a commit only needs the K/V of every layer
         launch_attention<TS>(c, nf, l);
-        EpiGateRes<TS> eo{sp, (const TS *)c->b_o[l], c->z, modl + 2 * d, mod_row, D};
+        EpiGateRes<TS> eo{sp, (const TS *)c->b_o[l], c->z, modl + 2 * d, mod_row, D,
+                          fold ? (TS *)c->hbuf : (TS *)nullptr, modl + 4 * d, fold ? c->ln_stats : (float2 *)nullptr};
         c->cls = CLS_GEMM_O;
         launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES, c->w_fc1[l],
-                        (size_t)d * D.dm);
-        c->cls = CLS_ADALN;
-        PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row,
-                (size_t)3 * d, (size_t)4 * d);
-        EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm};
+                        (size_t)d * D.dm, fold);
+        if (!fold) {
+            c->cls = CLS_ADALN;
+            PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row,
+                    (size_t)3 * d, (size_t)4 * d);
+        }
+        EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm, lm};
         c->cls = CLS_GEMM_FC1;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU, c->w_fc2[l],
-                        (size_t)d * D.dm);
-        EpiGateRes<TS> e2{sp, (const TS *)c->b_fc2[l], c->z, modl + 5 * d, mod_row, D};
+                        (size_t)d * D.dm, fold);
+        // the last layer's output goes to the final adaLN kernel, which reads z itself
+        const bool more = fold && l + 1 < L;
+        EpiGateRes<TS> e2{sp, (const TS *)c->b_fc2[l], c->z, modl + 5 * d, mod_row, D,
+                          more ? (TS *)c->hbuf : (TS *)nullptr, modl + 6 * d + d, more ? c->ln_stats : (float2 *)nullptr};
         c->cls = CLS_GEMM_FC2;
         launch_gemm<TS>(c, (const TS *)c->mbuf, (const TS *)c->w_fc2[l], M, d, D.dm, e2, TC_RES,
-                        l + 1 < L ? c->w_qkv[l + 1] : nullptr, (size_t)3 * d * d);
+                        l + 1 < L ? c->w_qkv[l + 1] : nullptr, (size_t)3 * d * d, fold);
     }
     if (kind == 0) {
         c->cls = CLS_HEAD;
@@ -377,7 +416,7 @@ static int run_pass_inner(nfd_ctx *c) {
         CK(c->launch_err);
         return NFD_OK;
     }
-    const int key = kind * 64 + nf + (c->fast ? 0 : 4096) + (c->h_sp.nc > 0 ? 0 : 8192);   // no conditioning kernels when all pairs are cached
+    const int key = kind * 64 + nf + (c->fast ? 0 : 4096) + (c->h_sp.nc > 0 ? 0 : 8192) + (c->fuse_ln ? 0 : 16384);   // no conditioning kernels when all pairs are cached
     auto it = c->graphs.find(key);
     if (it == c->graphs.end()) {
         GraphEntry ge;
@@ -580,6 +619,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     c->pend_act.assign(cfg->n_streams, std::vector<int>());
     if (getenv("NFD_NO_GRAPH")) c->use_graph = false;
     if (getenv("NFD_NO_FAST")) c->fast = false;
+    if (getenv("NFD_NO_FUSE_LN")) c->fuse_ln = false;
 
     int rc = c->bf16_mode ? repack_all<bf16>(c, w) : repack_all<float>(c, w);
     const int NF = NFD_MAX_PASS_FRAMES;
@@ -600,6 +640,10 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     c->cond_slots.assign(n_slots, nfd_ctx::CondSlot());
     A((void **)&c->mod, (size_t)n_slots * D.L * 6 * D.d * 4);
     A((void **)&c->fmod, (size_t)n_slots * 2 * D.d * 4);
+    if (c->bf16_mode) {
+        A((void **)&c->uvtab, (size_t)n_slots * D.L * (3 * D.d + D.dm) * sizeof(float2));
+        A((void **)&c->ln_stats, Mmax * ((D.d + 31) / 32) * sizeof(float2));
+    }
     A((void **)&c->pend_x0, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);
     A((void **)&c->pend_cz, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);
     A((void **)&c->xp, (size_t)NF * c->frame_elems() * 4);
@@ -616,6 +660,10 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
         if (rc == NFD_OK) { v = {c->w_t1, c->b_t1}; rc = upload_ptrs(c, v, &c->dp_t1); }
         if (rc == NFD_OK) { v = {c->w_t2, c->b_t2}; rc = upload_ptrs(c, v, &c->dp_t2); }
         if (rc == NFD_OK) { v = {c->w_fmod, c->b_fmod}; rc = upload_ptrs(c, v, &c->dp_fmod); }
+        if (rc == NFD_OK) { v = c->w_qkv; rc = upload_ptrs(c, v, &c->dp_wqkv); }
+        if (rc == NFD_OK) { v = c->b_qkv; rc = upload_ptrs(c, v, &c->dp_bqkv); }
+        if (rc == NFD_OK) { v = c->w_fc1; rc = upload_ptrs(c, v, &c->dp_wfc1); }
+        if (rc == NFD_OK) { v = c->b_fc1; rc = upload_ptrs(c, v, &c->dp_bfc1); }
     }
     if (rc == NFD_OK) {
         RopeTab rt;
@@ -1022,8 +1070,11 @@ int nfd_set_option(nfd_ctx *c, const char *name, int value) {
         c->use_graph = value != 0;
         return NFD_OK;
     }
-    if (!strcmp(name, "fast")) {
-        c->fast = value != 0;
+    if (!strcmp(name, "fast") || !strcmp(name, "fuse_ln")) {
+        // cached modulation rows carry the folded-LayerNorm vectors only if they were filled while the
+        // fold was active: start the cache afresh
+        (name[1] == 'a' ? c->fast : c->fuse_ln) = value != 0;
+        for (auto &cs : c->cond_slots) cs = nfd_ctx::CondSlot();
         return NFD_OK;
     }
     if (!strcmp(name, "lazy_commit")) {

@@ -160,6 +160,37 @@ __device__ __forceinline__ float warp_sum(float v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
+
+// Folded LayerNorm (see k_modw and the GEMM epilogues): what a GEMM that follows an adaLN needs in order to
+// apply the normalisation in its epilogue.
+struct LnFold {
+    const float2 *uv;       // (u, v) of this layer's projection: uv[slot * row_stride + n]; nullptr = not folded
+    size_t row_stride;
+    const float2 *stats;    // [rows][npart] (sum z, sum z^2) per 32 columns
+    int npart;              // d / 32
+    int norm;               // 0 LayerNorm, 1 RMSNorm
+    float eps;
+    const StepParams *sp;   // frame -> cache slot
+    int T;                  // rows per frame
+    static constexpr int kMaxFrames = 16;   // frames that a 128-row tile may span (the caller guarantees it)
+    __device__ __forceinline__ bool on() const { return uv != nullptr; }
+    // (u, v) of columns n, n+1 for the rows of frame j of the pass
+    __device__ __forceinline__ float4 uv_pair(int j, int n) const {
+        return *reinterpret_cast<const float4 *>(uv + (size_t)sp->fr[j].cond_row * row_stride + n);
+    }
+    // Row statistics are gathered by 8 adjacent lanes per row: lane `sub` takes partials sub, sub+8, ...
+    // (part), the lanes' sums are combined by a fixed shuffle tree and finished by finish().  The order of
+    // the additions depends on npart only, not on how the producer or the consumer tiled the rows.
+    __device__ __forceinline__ float2 part(int m, int i) const {
+        return (m >= 0 && i < npart) ? stats[(size_t)m * npart + i] : make_float2(0.f, 0.f);
+    }
+    __device__ __forceinline__ float2 finish(float s, float q) const {
+        const float inv_d = 1.0f / (float)(npart * 32);
+        const float mean = norm == 0 ? s * inv_d : 0.f;
+        const float var = fmaxf(q * inv_d - mean * mean, 0.f);
+        return make_float2(mean, rsqrtf(var + eps));
+    }
+};
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));

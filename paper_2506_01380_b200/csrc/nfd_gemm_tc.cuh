@@ -38,7 +38,8 @@ template <int BN> struct GemmCfg {
     static constexpr int SROW = BN + 4;                        // staging row stride (floats)
     static constexpr int STAGE_BYTES = 128 * SROW * 4;         // partial accumulator tile; reuses the ring
     static constexpr int TMEM_COLS = BN <= 32 ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
-    static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int UV_BYTES = LnFold::kMaxFrames * BN * 8;   // folded LayerNorm: (u, v) per frame and column
+    static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 1024 /*row statistics*/ + UV_BYTES;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
     static constexpr int MAX_S = 4;                            // largest cluster split
@@ -70,6 +71,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + G::STAGES),
                    accf = smem_u32(bars + 2 * G::STAGES);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * G::STAGES + 1);
+    float2 *rowstat = reinterpret_cast<float2 *>(smem + G::RING_BYTES + 256);   // (mean, rstd) of the tile's rows
+    float4 *uvs = reinterpret_cast<float4 *>(smem + G::RING_BYTES + 256 + 1024); // (u, v): [frame of the tile][BN]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb_all = (K + 63) / 64;
     const int kb0 = (int)((long long)nkb_all * split / S), kb1 = (int)((long long)nkb_all * (split + 1) / S);
@@ -101,6 +104,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const int n_items = rows_per * CPR;                      // items of this CTA's row slice
     const int r_base = (S > 1 ? (int)cluster_ctarank() : 0) * rows_per;   // first tile row of the slice
     typename Epi::Side side[MAX_ITEMS];
+    int uv_f0 = 0;                                           // first frame of the tile (folded LayerNorm)
+    if constexpr (Epi::kRowStats) uv_f0 = m0 / epi.ln.T;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -166,6 +171,49 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 if (m < M && n < N) epi.load(m, n, side[i]);
             }
         }
+        if constexpr (Epi::kRowStats) {
+            if (epi.ln.on()) {
+                // folded LayerNorm: (u, v) of the tile's columns for every frame the tile's rows belong to, and
+                // (mean, rstd) of the rows this CTA finishes, from the producer's partial sums
+                const int m_last = (m0 + 127 < M ? m0 + 127 : M - 1);
+                const int n_fr = m_last / epi.ln.T - uv_f0 + 1;
+                for (int idx = et; idx < n_fr * (BN / 2); idx += G::EPI_THREADS) {
+                    const int fr = idx / (BN / 2), c2 = idx - fr * (BN / 2);
+                    if (n0 + 2 * c2 < N) uvs[idx] = epi.ln.uv_pair(uv_f0 + fr, n0 + 2 * c2);
+                }
+                // 8 lanes per row, 32 rows per sweep; every load is issued before the first sum
+                constexpr int SWEEPS = 128 / (G::EPI_THREADS / 8);
+                const int sub = et & 7;
+                float2 pv[SWEEPS][4];
+#pragma unroll
+                for (int w = 0; w < SWEEPS; ++w) {
+                    const int r = (et >> 3) + w * (G::EPI_THREADS / 8);
+                    const int m = (r < rows_per && m0 + r_base + r < M) ? m0 + r_base + r : -1;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) pv[w][u] = epi.ln.part(m, sub + 8 * u);
+                }
+#pragma unroll
+                for (int w = 0; w < SWEEPS; ++w) {
+                    const int r = (et >> 3) + w * (G::EPI_THREADS / 8);
+                    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) s1 += pv[w][u].x, s2 += pv[w][u].y;
+                    if (epi.ln.npart > 32) {              // rows wider than 1024
+                        const int m = (r < rows_per && m0 + r_base + r < M) ? m0 + r_base + r : -1;
+                        for (int i = sub + 32; i < epi.ln.npart; i += 8) {
+                            const float2 t = epi.ln.part(m, i);
+                            s1 += t.x, s2 += t.y;
+                        }
+                    }
+#pragma unroll
+                    for (int o = 1; o < 8; o <<= 1) {
+                        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+                        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+                    }
+                    if (sub == 0 && r < rows_per) rowstat[r_base + r] = epi.ln.finish(s1, s2);
+                }
+            }
+        }
         // partial accumulator: tensor memory -> this CTA's staging tile (the ring is free by now)
         const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;                    // which half of the columns
@@ -200,6 +248,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const uint32_t stage_u32 = smem_u32(stage);
         for (int i0 = 0; i0 * G::EPI_THREADS < n_items; i0 += MAX_ITEMS) {
             int mm[MAX_ITEMS], nn[MAX_ITEMS], tr[MAX_ITEMS];
+            unsigned vmask[MAX_ITEMS];
 #pragma unroll
             for (int i = 0; i < MAX_ITEMS; ++i) {
                 const int it = et + (i0 + i) * G::EPI_THREADS;
@@ -209,6 +258,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     mm[i] = -1;
                 else if (i0 > 0)
                     epi.load(mm[i], nn[i], side[i]);
+                vmask[i] = __ballot_sync(0xffffffffu, mm[i] >= 0);
             }
 #pragma unroll
             for (int j0 = 0; j0 < MAX_ITEMS; j0 += 2) {
@@ -244,8 +294,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                         }
                     }
                     float a[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                    epi.apply(mm[i], nn[i], a, side[i]);
+                    float2 ms = make_float2(0.f, 1.f);
+                    const float4 *uvp = nullptr;
+                    if constexpr (Epi::kRowStats) {
+                        if (epi.ln.on()) {
+                            ms = rowstat[tr[i]];
+                            uvp = uvs + ((mm[i] / epi.ln.T - uv_f0) * BN + (nn[i] - n0)) / 2;
+                        }
+                    }
+                    epi.apply(mm[i], nn[i], a, side[i], ms, uvp, vmask[i]);
                 }
+                if (i0 == 0 && j0 == 0) NFD_TRACE_MARK_T(TRK_OTHER + 7, 64);
             }
         }
     }

@@ -122,17 +122,88 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
 }
 
 // ---------------------------------------------------------------------------
+// Folded LayerNorm, weight side.  A projection that follows an adaLN,
+//     y[n] = sum_k ((z[k] - mean) * rstd * (1 + scale[k]) + shift[k]) * W[n][k] + b[n],
+// equals
+//     y[n] = rstd * (sum_k z[k] (1 + scale[k]) W[n][k]  -  mean * u[n]) + v[n],
+//     u[n] = sum_k (1 + scale[k]) W[n][k],      v[n] = sum_k shift[k] W[n][k] + b[n],
+// so the GEMM can run on z*(1+scale), written by the kernel that produces z,
+// and apply mean and rstd per row in its epilogue.  u and v depend on the
+// conditioning row only and are kept in the modulation cache next to shift and
+// scale.  This kernel fills (u, v) for the QKV projection (outputs 0..3d) and
+// the first MLP projection (outputs 3d..3d+dm) of layer blockIdx.y, one warp
+// per output, four conditioning rows at a time.
+// ---------------------------------------------------------------------------
+template <typename TS>
+__global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *const *Wqkv_l, const TS *const *bqkv_l,
+                                              const TS *const *Wfc1_l, const TS *const *bfc1_l, const float *mod,
+                                              size_t mod_row_stride, float2 *uv, size_t uv_row_stride, int d, int dm) {
+    NFD_TRACE_T0();
+    pdl_wait();
+    pdl_launch();
+    constexpr int NV = WVec<TS>::N;
+    const int layer = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int o = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (o >= 3 * d + dm) return;
+    const bool mlp = o >= 3 * d;
+    const int oo = mlp ? o - 3 * d : o;
+    const TS *wrow = (mlp ? Wfc1_l[layer] : Wqkv_l[layer]) + (size_t)oo * d;
+    const float bo = to_f((mlp ? bfc1_l[layer] : bqkv_l[layer])[oo]);
+    const size_t off_shift = (size_t)layer * 6 * d + (mlp ? 3 * d : 0);
+    const size_t off_scale = off_shift + d;
+    const int nc = sp->nc;
+    for (int c0 = 0; c0 < nc; c0 += 4) {
+        float au[4] = {0.f, 0.f, 0.f, 0.f}, av[4] = {0.f, 0.f, 0.f, 0.f};
+        const float *mrow[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) mrow[r] = mod + (size_t)sp->cd[c0 + r < nc ? c0 + r : c0].slot * mod_row_stride;
+        for (int i = lane * NV; i < d; i += 32 * NV) {
+            float w[NV];
+            WVec<TS>::load(wrow + i, w);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                if (c0 + r < nc) {
+#pragma unroll
+                    for (int e = 0; e < NV; e += 4) {
+                        const float4 sc = *reinterpret_cast<const float4 *>(mrow[r] + off_scale + i + e);
+                        const float4 sh = *reinterpret_cast<const float4 *>(mrow[r] + off_shift + i + e);
+                        au[r] = fmaf(w[e], 1.0f + sc.x, au[r]), av[r] = fmaf(w[e], sh.x, av[r]);
+                        au[r] = fmaf(w[e + 1], 1.0f + sc.y, au[r]), av[r] = fmaf(w[e + 1], sh.y, av[r]);
+                        au[r] = fmaf(w[e + 2], 1.0f + sc.z, au[r]), av[r] = fmaf(w[e + 2], sh.z, av[r]);
+                        au[r] = fmaf(w[e + 3], 1.0f + sc.w, au[r]), av[r] = fmaf(w[e + 3], sh.w, av[r]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            if (c0 + r >= nc) break;
+            const float su = warp_sum(au[r]), sv = warp_sum(av[r]);
+            if (lane == 0)
+                uv[(size_t)sp->cd[c0 + r].slot * uv_row_stride + (size_t)layer * (3 * d + dm) + o] =
+                    make_float2(su, sv + bo);
+        }
+    }
+    NFD_TRACE_END(TRK_GEMV);
+}
+
+// ---------------------------------------------------------------------------
 // Patchify + embed: z[tok][o] = sum_p (alpha*x_a + beta*x_b)[patch p of tok] * W_pe[p][o] + b[o].
 // A CTA takes PE_TOK tokens (blockIdx.x) and 256 output columns (blockIdx.y).
 // Each thread owns one output column: it loads 64 rows of its W_pe column at a
 // time into registers (independent loads, all in flight together) and reuses
 // them for all tokens of the CTA.  W_pe is used in its [P][d] layout so that
 // adjacent threads read adjacent columns.
+// With a_out set (folded LayerNorm, see the GEMM epilogues below; d a multiple of
+// 32) it also writes the first layer's GEMM operand z*(1+scale) and the row-sum
+// partials of z per 32 columns.
 // ---------------------------------------------------------------------------
 #define PE_TOK 16
 template <typename TS>
 __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
-                                                     float *z) {
+                                                     float *z, TS *a_out, float2 *stats, const float *scale0,
+                                                     size_t mod_row_stride) {
     extern __shared__ float s_patch[];          // [PE_TOK][P]
     NFD_TRACE_T0();
     pdl_wait();
@@ -188,8 +259,18 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
     }
     const float bo = to_f(b_pe[o]);
 #pragma unroll
-    for (int t = 0; t < PE_TOK; ++t)
-        if (m0 + t < M) z[(size_t)(m0 + t) * D.d + o] = acc[t] + bo;
+    for (int t = 0; t < PE_TOK; ++t) {
+        if (m0 + t >= M) break;
+        const int m = m0 + t;
+        const float zv = acc[t] + bo;
+        z[(size_t)m * D.d + o] = zv;
+        if (a_out) {
+            const float sc = scale0[(size_t)sp->fr[m / D.T].cond_row * mod_row_stride + o];
+            a_out[(size_t)m * D.d + o] = from_f<TS>(zv * (1.0f + sc));
+            const float s1 = warp_sum(zv), s2 = warp_sum(zv * zv);
+            if ((threadIdx.x & 31) == 0) stats[(size_t)m * (D.d >> 5) + (o >> 5)] = make_float2(s1, s2);
+        }
+    }
     NFD_TRACE_END(TRK_PATCH);
 }
 
@@ -333,8 +414,31 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float *f) {
 // of 8, 16 bytes at a time, in two steps: load() fetches everything the item
 // needs besides the accumulators (bias, gate, residual, rotary table) into a
 // Side record, so that the fetch can be issued while the UMMAs still run;
-// apply() combines it with the accumulators and stores.
+// apply() combines it with the accumulators and stores.  apply() also gets the
+// (mean, rstd) of the item's row and the (u, v) pairs of its 8 columns (in shared
+// memory) when the functor asks for row statistics (kRowStats) and the
+// LayerNorm is folded, and the mask of the warp's lanes that hold a valid item; four
+// adjacent lanes always hold the four 8-column items of one 32-column group.
+//
+// Folded LayerNorm (tensor-core path only, see k_modw): the functors that update
+// the residual stream z also write the next GEMM's operand z*(1+scale) and the
+// (sum z, sum z^2) partials of every 32 columns of the row; the functors of the
+// GEMMs that follow an adaLN turn those partials into (mean, rstd) and apply
+// rstd*(acc - mean*u[n]) + v[n].
 // ---------------------------------------------------------------------------
+__device__ __forceinline__ void ln_fold_apply(float *a, const float4 *uv, float2 ms) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        a[2 * i] = fmaf(ms.y, fmaf(-ms.x, uv[i].x, a[2 * i]), uv[i].y);
+        a[2 * i + 1] = fmaf(ms.y, fmaf(-ms.x, uv[i].z, a[2 * i + 1]), uv[i].w);
+    }
+}
+__device__ __forceinline__ void bias_add(float *a, const uint4 &bits) {
+    float b[8];
+    unpack_bf16x8(bits, b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] += b[i];
+}
 // QKV: + bias, 3D RoPE on q and k (Section 3.1 "3D Positional Embedding":
 // adjacent pairs, per-axis frequencies), q -> [H][Nq][dh], k/v -> cache pages.
 template <typename TS> struct EpiQKV {
@@ -346,6 +450,7 @@ template <typename TS> struct EpiQKV {
     int layer;
     const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by the tensor-core path
     int n_rows;                 // nf*T: rows of the pass (q is [H][n_rows][dh])
+    LnFold ln;                  // folded adaLN in front of this projection (tensor-core path only)
     // Pull the cached K/V pages that the attention kernel of this layer is about to read towards L2 (the
     // pages of frames before this pass are final); each CTA of the launch takes a slice of every page.
     __device__ __forceinline__ void prefetch(unsigned int cta, unsigned int n_cta) const {
@@ -363,30 +468,32 @@ template <typename TS> struct EpiQKV {
         }
     }
     static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
+    static constexpr bool kRowStats = true;
     struct Side {
-        uint4 bias;
+        uint4 bias;             // unused with the folded LayerNorm (v carries the bias)
         float4 c01, c23;        // (cos, sin) of four adjacent pairs
         int stream, frame;      // of the token's frame
     };
     __device__ __forceinline__ void load(int m, int n, Side &s) const {
-        s.bias = *reinterpret_cast<const uint4 *>(bias + n);
+        const FrameDesc &f = sp->fr[m / D.T];
+        if (!ln.on()) s.bias = *reinterpret_cast<const uint4 *>(bias + n);
         const int which = n / D.d, col = n - which * D.d;
         const int e = col % D.dh;
         if (which < 2) {
             const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
             s.c01 = cs[0], s.c23 = cs[1];
         }
-        const FrameDesc &f = sp->fr[m / D.T];
         s.stream = f.stream, s.frame = f.frame;
     }
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
-        float b[8];
-        unpack_bf16x8(s.bias, b);
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2 ms, const float4 *uv,
+                                          unsigned) const {
         const int which = n / D.d, col = n - which * D.d;
         const int head = col / D.dh, e = col - head * D.dh;
         const int j = m / D.T, tok = m - j * D.T;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] += b[i];
+        if (ln.on())
+            ln_fold_apply(a, uv, ms);
+        else
+            bias_add(a, s.bias);
         TS *dst;
         if (which < 2) {
             const float cv[4] = {s.c01.x, s.c01.z, s.c23.x, s.c23.z}, sv[4] = {s.c01.y, s.c01.w, s.c23.y, s.c23.w};
@@ -435,7 +542,9 @@ template <typename TS> struct EpiQKV {
     }
 };
 
-// z += gate_f * (acc + bias): residual update of the fp32 stream.
+// z += gate_f * (acc + bias): residual update of the fp32 stream.  With stats set
+// (folded LayerNorm) it also writes the row-sum partials of the new z and, with
+// a_out set, the next GEMM's operand z*(1+scale_next).
 template <typename TS> struct EpiGateRes {
     const StepParams *sp;
     const TS *bias;
@@ -443,11 +552,15 @@ template <typename TS> struct EpiGateRes {
     const float *gate;      // mod + layer offset + chunk offset
     size_t row_stride;
     Dims D;
+    TS *a_out;              // [rows][d] or nullptr
+    const float *scale_next;// mod + layer offset + chunk offset of the adaLN scale that follows (with a_out)
+    float2 *stats;          // [rows][d/32] or nullptr
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 2;        // epilogue items a thread keeps in flight together
+    static constexpr bool kRowStats = false;
     struct Side {
         uint4 bias;
-        float4 g0, g1, z0, z1;
+        float4 g0, g1, z0, z1, s0, s1;
     };
     __device__ __forceinline__ void load(int m, int n, Side &s) const {
         s.bias = *reinterpret_cast<const uint4 *>(bias + n);
@@ -456,8 +569,13 @@ template <typename TS> struct EpiGateRes {
         const float4 *zp = reinterpret_cast<const float4 *>(z + (size_t)m * D.d + n);
         s.g0 = g[0], s.g1 = g[1];
         s.z0 = zp[0], s.z1 = zp[1];
+        if (a_out) {
+            const float4 *sc = reinterpret_cast<const float4 *>(scale_next + (size_t)row * row_stride + n);
+            s.s0 = sc[0], s.s1 = sc[1];
+        }
     }
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2, const float4 *,
+                                          unsigned mask) const {
         float b[8];
         unpack_bf16x8(s.bias, b);
         float4 z0 = s.z0, z1 = s.z1;
@@ -472,6 +590,21 @@ template <typename TS> struct EpiGateRes {
         float4 *zp = reinterpret_cast<float4 *>(z + (size_t)m * D.d + n);
         zp[0] = z0;
         zp[1] = z1;
+        if (stats) {
+            if (a_out) {
+                float o[8] = {z0.x * (1.0f + s.s0.x), z0.y * (1.0f + s.s0.y), z0.z * (1.0f + s.s0.z),
+                              z0.w * (1.0f + s.s0.w), z1.x * (1.0f + s.s1.x), z1.y * (1.0f + s.s1.y),
+                              z1.z * (1.0f + s.s1.z), z1.w * (1.0f + s.s1.w)};
+                *reinterpret_cast<uint4 *>(a_out + (size_t)m * D.d + n) = pack_bf16x8(o);
+            }
+            // the four lanes of a 32-column group hold the same row and are valid together
+            float s1 = ((z0.x + z0.y) + (z0.z + z0.w)) + ((z1.x + z1.y) + (z1.z + z1.w));
+            float s2 = ((z0.x * z0.x + z0.y * z0.y) + (z0.z * z0.z + z0.w * z0.w)) +
+                       ((z1.x * z1.x + z1.y * z1.y) + (z1.z * z1.z + z1.w * z1.w));
+            s1 += __shfl_xor_sync(mask, s1, 1), s2 += __shfl_xor_sync(mask, s2, 1);
+            s1 += __shfl_xor_sync(mask, s1, 2), s2 += __shfl_xor_sync(mask, s2, 2);
+            if ((n & 31) == 0) stats[(size_t)m * (D.d >> 5) + (n >> 5)] = make_float2(s1, s2);
+        }
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
         const int row = sp->fr[m / D.T].cond_row;
@@ -487,20 +620,25 @@ template <typename TS> struct EpiGelu {
     const TS *bias;
     TS *out;
     int N;
+    LnFold ln;              // folded adaLN in front of this projection (tensor-core path only)
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 8;        // epilogue items a thread keeps in flight together
+    static constexpr bool kRowStats = true;
     struct Side {
-        uint4 bias;
+        uint4 bias;         // unused with the folded LayerNorm (v carries the bias)
     };
     __device__ __forceinline__ void load(int m, int n, Side &s) const {
         (void)m;
-        s.bias = *reinterpret_cast<const uint4 *>(bias + n);
+        if (!ln.on()) s.bias = *reinterpret_cast<const uint4 *>(bias + n);
     }
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s) const {
-        float b[8];
-        unpack_bf16x8(s.bias, b);
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2 ms, const float4 *uv,
+                                          unsigned) const {
+        if (ln.on())
+            ln_fold_apply(a, uv, ms);
+        else
+            bias_add(a, s.bias);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i] + b[i]);
+        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i]);
         *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
@@ -517,11 +655,13 @@ template <typename TS> struct EpiFinal {
     Dims D;
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
+    static constexpr bool kRowStats = false;
     struct Side {
         int unused;
     };
     __device__ __forceinline__ void load(int, int, Side &) const {}
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &) const {
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &, float2, const float4 *,
+                                          unsigned) const {
 #pragma unroll
         for (int i = 0; i < 8; i += 2) (*this)(m, n + i, a[i], a[i + 1]);
     }

@@ -75,6 +75,8 @@ CASES = [
     ("tiny_bf16", "stress", {"fast": 0}),
     ("tiny_bf16", "paper", {}),
     ("tiny_bf16", "stress", {}),
+    ("tiny_bf16", "paper", {"fuse_ln": 0}),       # in-layer adaLN as kernels of their own
+    ("tiny_bf16", "stress", {"fuse_ln": 0}),
 ]
 
 
@@ -248,8 +250,8 @@ def test_attention_alone(n_kv, n_q, window, fast):
     assert g.status() == 0
 
 
-def _teacher_forced(cfg, kind, n_prompt, k, seed):
-    g, orc = make_pair(cfg, seed, kind)
+def _teacher_forced(cfg, kind, n_prompt, k, seed, **opts):
+    g, orc = make_pair(cfg, seed, kind, **opts)
     prompt(cfg, g, orc, n_prompt, seed=700 + seed, group=4)
     x_t = I.round_bf16(I.make_latents(cfg, k, 800 + seed))
     t = float(np.float32(O.fm_time(3 * math.pi / 8)))
@@ -267,8 +269,11 @@ def _teacher_forced(cfg, kind, n_prompt, k, seed):
 
 
 @pytest.mark.parametrize("kind", ["paper", "stress"])
-def test_310m_slice_two_layers(kind):
-    _teacher_forced(I.make_cfg("nfd310m_slice"), kind, n_prompt=5, k=2, seed=0)
+@pytest.mark.parametrize("fuse_ln", [1, 0])
+def test_310m_slice_two_layers(kind, fuse_ln):
+    """Two layers at model width, with the in-layer LayerNorms folded into the neighbouring GEMMs (the
+    default) and as kernels of their own."""
+    _teacher_forced(I.make_cfg("nfd310m_slice"), kind, n_prompt=5, k=2, seed=0, fuse_ln=fuse_ln)
 
 
 def test_310m_full_config_teacher_forced():
@@ -295,7 +300,7 @@ def test_modulation_cache_hits_evictions_and_values():
     assert torch.equal(v_first, v_again)
     check(v_first, orc.denoise_step(x.cpu().numpy().astype(np.float64), 0.625, 3), cfg["dtype"], "velocity")
     # more distinct pairs than the cache has slots: the first pair is replaced ...
-    for i in range(120):
+    for i in range(300):
         g.denoise_step(x, float(np.float32(0.001 * (i + 1))), i % cfg["n_actions"])
     h1, m1 = g.cond_cache_stats()
     v_refill = g.denoise_step(x, 0.625, 3).clone()
