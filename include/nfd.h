@@ -239,6 +239,17 @@ int nfd_profile_end(nfd_ctx *ctx, int n_classes, long long *n_launches, float *t
 int nfd_profile_class_count(void);
 const char *nfd_profile_class_name(int id);
 
+/* Fills the modulation cache for every (time, action) pair that nfd_speculate
+ * and the commits can ask for: the n_steps sampler times (Section 4.1
+ * "Sampling") and the context time (Section 4.3), each with every action.  The
+ * adaLN modulation depends on nothing else (Section 3.1 "Action Conditioning"),
+ * so after this call a generation loop runs no conditioning kernels at all.
+ * Returns the number of pairs computed (pairs already cached are left alone),
+ * NFD_E_RANGE if (n_steps + 1) * n_actions exceeds the cache's 256 rows (nothing
+ * is done then: the cache keeps working on demand), or another negative code.
+ * Asynchronous on the context's stream. */
+int nfd_warm_modulation(nfd_ctx *ctx);
+
 /* Run-time switches, for tests and profiling: "graph" 0/1 (replay CUDA graphs
  * or launch kernels directly), "fast" 0/1 (tensor-core kernels or the plain
  * validation kernels; bf16 only), "lazy_commit" 0/1 (defer the commit of

@@ -301,17 +301,17 @@ template <typename TS> static void launch_attention(nfd_ctx *c, int nf, int laye
                 (const TS *)c->kc, (const TS *)c->vc, (TS *)c->abuf);
 }
 
-// Kernels after k_set_params.  nf and kind are fixed per captured graph.
-template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
+// Conditioning kernels for the c->h_sp.nc (time, action) pairs that the pass found missing in the
+// modulation cache; `rows` bounds their number (grid of the embedding kernel).
+template <typename TS> static void enqueue_conditioning(nfd_ctx *c, int rows) {
     const Dims &D = c->D;
-    const int d = D.d, L = D.L, M = nf * D.T;
+    const int d = D.d, L = D.L, nf = rows;
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
     const size_t uv_row = (size_t)L * (3 * d + D.dm);
     const bool fold = c->fold_active();
-    // conditioning: only for the (t, action) pairs that are not in the modulation cache
     c->cls = CLS_COND;
-    if (c->h_sp.nc > 0) {
+    {
         PLAUNCH(c, k_temb, nf, 128, 0, sp, D.t_scale, c->emb);
         PLAUNCH(c, (k_gemv<TS, GEMV_T1>), dim3((d + 7) / 8, 1), 256, 0, sp, (const TS *const *)c->dp_t1,
                 (const TS *const *)(c->dp_t1 + 1), (const TS *)nullptr, (const float *)c->emb, c->h1, 256, d, (size_t)d,
@@ -330,6 +330,18 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
                     (const TS *const *)c->dp_bqkv, (const TS *const *)c->dp_wfc1, (const TS *const *)c->dp_bfc1,
                     (const float *)c->mod, mod_row, c->uvtab, uv_row, d, D.dm);
     }
+}
+
+// Kernels after k_set_params.  nf and kind are fixed per captured graph.
+template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
+    const Dims &D = c->D;
+    const int d = D.d, L = D.L, M = nf * D.T;
+    const StepParams *sp = c->d_sp;
+    const size_t mod_row = (size_t)L * 6 * d;
+    const size_t uv_row = (size_t)L * (3 * d + D.dm);
+    const bool fold = c->fold_active();
+    // conditioning: only for the (t, action) pairs that are not in the modulation cache
+    if (c->h_sp.nc > 0) enqueue_conditioning<TS>(c, nf);
     // tokens
     c->cls = CLS_PATCH;
     if (c->bf16_mode && c->fast)
@@ -746,6 +758,59 @@ static void commit_coeffs(const nfd_ctx *c, float *t_fm, float *a, float *b) {
     const double t = sn / (sn + cs);
     const double scale = sqrt(t * t + (1 - t) * (1 - t));
     *t_fm = (float)t, *a = (float)(cs * scale / sd), *b = (float)(sn * scale);
+}
+
+// FM time of sampler step s (Section 4.1 "Sampling": t' from pi/2 down in S equal steps).
+static double sampler_fm_time(int S, int s) {
+    const double tp = 0.5 * M_PI * (double)(S - s) / (double)S;
+    const double sn = sin(tp), cs = cos(tp);
+    return sn / (sn + cs);
+}
+
+// Fill the modulation cache for every (time, action) pair that nfd_speculate and the commits can ask for:
+// the S sampler times and the context time, for each action.  Pairs that are cached already are left alone.
+int nfd_warm_modulation(nfd_ctx *c) {
+    if (!c) return NFD_E_NULLPTR;
+    const int S = c->cfg.n_steps, A = c->cfg.n_actions;
+    std::vector<float> ts;
+    for (int s = 0; s < S; ++s) ts.push_back((float)sampler_fm_time(S, s));
+    float t_fm, ca, cb;
+    commit_coeffs(c, &t_fm, &ca, &cb);
+    ts.push_back(t_fm);
+    if ((long long)ts.size() * A > (long long)c->cond_slots.size()) return NFD_E_RANGE;
+    int filled = 0;
+    std::vector<std::pair<float, int>> todo;
+    for (float t : ts)
+        for (int a = 0; a < A; ++a) todo.push_back(std::make_pair(t, a));
+    for (size_t i0 = 0; i0 < todo.size(); i0 += NFD_MAX_PASS_FRAMES) {
+        // a conditioning-only pass: the frame list is only used to look the pairs up
+        std::vector<PassFrame> fr;
+        for (size_t i = i0; i < todo.size() && i < i0 + NFD_MAX_PASS_FRAMES; ++i) {
+            PassFrame f;
+            f.stream = 0, f.frame = 0, f.t = todo[i].first, f.action = todo[i].second, f.first_new = 0;
+            f.src = 0, f.src_index = 0, f.out_index = -1;
+            fr.push_back(f);
+        }
+        RET(build_pass_frames(c, fr, 2, PassInputs()));
+        const int nc = c->h_sp.nc;
+        if (nc == 0) continue;
+        c->cls = CLS_PARAMS;
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        if (c->bf16_mode)
+            enqueue_conditioning<bf16>(c, (int)fr.size());
+        else
+            enqueue_conditioning<float>(c, (int)fr.size());
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess) e = c->launch_err;
+        if (e != cudaSuccess) {
+            c->launch_err = cudaSuccess;
+            for (int r = 0; r < nc; ++r) c->cond_slots[c->h_sp.cd[r].slot] = nfd_ctx::CondSlot();
+            fprintf(stderr, "libnfd: %s\n", cudaGetErrorString(e));
+            return NFD_E_CUDA;
+        }
+        filled += nc;
+    }
+    return filled;
 }
 
 // Commit pass over n streams x k frames; actions per frame.

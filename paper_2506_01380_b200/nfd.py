@@ -42,7 +42,8 @@ class NfdWeights(C.Structure):
 EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_denoise_step_at",
            "nfd_denoise_step_batched", "nfd_commit_frame", "nfd_speculate", "nfd_speculate_batched",
            "nfd_rollback", "nfd_kv_state", "nfd_kv_hash", "nfd_kv_read", "nfd_attention", "nfd_status",
-           "nfd_launch_count", "nfd_set_option", "nfd_strerror", "nfd_profile_begin", "nfd_profile_end",
+           "nfd_launch_count", "nfd_set_option", "nfd_warm_modulation", "nfd_strerror", "nfd_profile_begin",
+           "nfd_profile_end",
            "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc", "nfd_cond_cache_stats"]
 
 
@@ -82,6 +83,7 @@ def load():
     lib.nfd_launch_count.argtypes = [vp]
     lib.nfd_launch_count.restype = C.c_longlong
     lib.nfd_set_option.argtypes = [vp, C.c_char_p, C.c_int]
+    lib.nfd_warm_modulation.argtypes = [vp]
     lib.nfd_profile_begin.argtypes = [vp]
     lib.nfd_profile_end.argtypes = [vp, C.c_int, C.POINTER(C.c_longlong), fp]
     lib.nfd_profile_class_count.argtypes = []
@@ -321,6 +323,17 @@ class NFD:
         cnt, ms = (C.c_longlong * n)(), (C.c_float * n)()
         _check(self.lib.nfd_profile_end(self._h, n, cnt, ms), "nfd_profile_end")
         return {self.lib.nfd_profile_class_name(i).decode(): (int(cnt[i]), float(ms[i])) for i in range(n)}
+
+    def warm_modulation(self) -> int:
+        """Precompute the modulation of every (schedule time, action) pair; returns the number computed."""
+        self._enter()
+        try:
+            n = self.lib.nfd_warm_modulation(self._h)
+        finally:
+            self._exit()
+        if n < 0:
+            _check(n, "nfd_warm_modulation")
+        return n
 
     def set_option(self, name: str, value: int):
         _check(self.lib.nfd_set_option(self._h, name.encode(), int(value)), "nfd_set_option")

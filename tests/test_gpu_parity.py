@@ -313,6 +313,35 @@ def test_modulation_cache_hits_evictions_and_values():
     assert g.status() == 0
 
 
+@pytest.mark.parametrize("name", ["tiny_bf16", "tiny"])
+def test_warm_modulation_fills_every_schedule_pair(name):
+    """nfd_warm_modulation computes the modulation of all (sampler or context time, action) pairs up front:
+    a generation loop that follows finds every pair cached, and its frames and cache contents are bitwise
+    those of a context that computes the pairs on demand."""
+    from paper_2506_01380_b200.nfd import NFD
+    torch = _torch()
+    cfg = I.make_cfg(name)
+    w = I.make_weights(cfg, 11, "stress")
+    warm, cold = NFD(cfg, w), NFD(cfg, w)
+    n_pairs = (cfg["n_steps"] + 1) * cfg["n_actions"]
+    assert warm.warm_modulation() == n_pairs
+    assert warm.warm_modulation() == 0                      # all cached already
+    _, m0 = warm.cond_cache_stats()
+    fs = I.frame_shape(cfg)
+    for step in range(6):
+        k = 1 + step % 2
+        noise = dev(I.make_latents(cfg, cfg["n_steps"] * k, 40 + step).reshape((cfg["n_steps"], k) + fs))
+        cz = dev(I.make_latents(cfg, k, 60 + step))
+        a = (3 * step + 1) % cfg["n_actions"]
+        ya, yb = warm.speculate(k, a, noise, cz), cold.speculate(k, a, noise, cz)
+        assert torch.equal(ya, yb)
+        warm.rollback(k), cold.rollback(k)
+    assert warm.cond_cache_stats()[1] == m0, "no pair may be missing after the warm-up"
+    assert cold.cond_cache_stats()[1] > 0
+    assert warm.kv_hash() == cold.kv_hash()
+    assert warm.status() == 0 and cold.status() == 0
+
+
 @pytest.mark.parametrize("name", ["tiny_bf16", "tiny", "nfd310m_slice"])
 def test_deferred_commit_equals_immediate_commit(name):
     """A speculation leaves the commit of its frames to the first pass of the next speculation (the paper's
