@@ -96,27 +96,39 @@ __device__ __forceinline__ unsigned long long nfd_trace_now() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void nfd_trace_put(int kind, unsigned long long t0) {
-    const unsigned int i = atomicAdd(&g_trace_n, 1u);
-    if (i < NFD_TRACE_CAP) {
-        unsigned int sm;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
-        g_trace[i].t0 = t0, g_trace[i].t1 = nfd_trace_now(), g_trace[i].kind = kind, g_trace[i].sm = (int)sm;
+// Point events inside a kernel (NFD_TRACE_MARK*) are kept in shared memory and written out together with
+// the CTA's record at NFD_TRACE_END, so that taking a mark costs one shared-memory store and does not
+// disturb what it measures.  A mark must not be taken before the kernel's first __syncthreads().
+#define NFD_TRACE_MARKS 24
+__device__ __forceinline__ void nfd_trace_flush(int kind, unsigned long long t0, const unsigned long long *marks) {
+    int n = 1;
+    for (int i = 0; i < NFD_TRACE_MARKS; ++i) n += marks[i] != 0;
+    unsigned int at = atomicAdd(&g_trace_n, (unsigned int)n);
+    unsigned int sm;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+    sm |= (blockIdx.x & 0xfffu) << 8 | (blockIdx.y & 0xfffu) << 20;      // SM in bits 0-7, then blockIdx.x, .y
+    if (at < NFD_TRACE_CAP) g_trace[at].t0 = t0, g_trace[at].t1 = nfd_trace_now(), g_trace[at].kind = kind, g_trace[at].sm = (int)sm;
+    for (int i = 0; i < NFD_TRACE_MARKS; ++i) {
+        if (!marks[i]) continue;
+        ++at;
+        if (at < NFD_TRACE_CAP) g_trace[at].t0 = g_trace[at].t1 = marks[i], g_trace[at].kind = i, g_trace[at].sm = (int)sm;
     }
 }
-#define NFD_TRACE_T0() const unsigned long long nfd_t0_ = nfd_trace_now()
+#define NFD_TRACE_T0()                                               \
+    const unsigned long long nfd_t0_ = nfd_trace_now();              \
+    __shared__ unsigned long long nfd_marks_[NFD_TRACE_MARKS];       \
+    if (threadIdx.x < NFD_TRACE_MARKS) nfd_marks_[threadIdx.x] = 0
 #define NFD_TRACE_END(kind)                          \
     do {                                             \
-        if (threadIdx.x == 0) nfd_trace_put((kind), nfd_t0_); \
+        if (threadIdx.x == 0) nfd_trace_flush((kind), nfd_t0_, nfd_marks_); \
     } while (0)
-// a point event (t0 == t1 is the time of the call), e.g. right after the wait on the predecessor grid
 #define NFD_TRACE_MARK(kind)                                  \
     do {                                                      \
-        if (threadIdx.x == 0) nfd_trace_put((kind), nfd_trace_now()); \
+        if (threadIdx.x == 0) nfd_marks_[(kind) % NFD_TRACE_MARKS] = nfd_trace_now(); \
     } while (0)
 #define NFD_TRACE_MARK_T(kind, tid)                           \
     do {                                                      \
-        if (threadIdx.x == (tid)) nfd_trace_put((kind), nfd_trace_now()); \
+        if (threadIdx.x == (tid)) nfd_marks_[(kind) % NFD_TRACE_MARKS] = nfd_trace_now(); \
     } while (0)
 #else
 #define NFD_TRACE_T0() do { } while (0)

@@ -174,8 +174,11 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
         const double kb = (double)((nkb + S - 1) / S);
         const double load = kb * (16384.0 + BN * 128.0) / 55.0 * share;
         const double items = (128.0 / S) * (BN / 8.0) / 256.0;                 // epilogue items per thread
-        const double epi = 400.0 + items * 350.0 + (S - 1) * 900.0 + BN * 4.0;     // remote partials are slow to fetch
-        const double fixed = 3200.0 + (S > 1 ? 800.0 : 0.0);
+        // with S > 1 every pair of items waits for the partials of the S - 1 other CTAs (distributed shared
+        // memory: a slow round trip per pair, longer the more peers are asked)
+        const double pairs = (double)(((int)(items + 0.999) + 1) / 2);
+        const double epi = 400.0 + items * 350.0 + (S - 1) * (pairs * 1000.0 + 300.0) + BN * 4.0;
+        const double fixed = 3200.0 + (S > 1 ? 500.0 : 0.0);
         return waves * (fixed + load + epi);
     };
     const int bns[4] = {32, 64, 96, 128};

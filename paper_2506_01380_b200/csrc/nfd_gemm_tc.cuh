@@ -39,7 +39,9 @@ template <int BN> struct GemmCfg {
     static constexpr int STAGE_BYTES = 128 * SROW * 4;         // partial accumulator tile; reuses the ring
     static constexpr int TMEM_COLS = BN <= 32 ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
     static constexpr int UV_BYTES = LnFold::kMaxFrames * BN * 8;   // folded LayerNorm: (u, v) per frame and column
-    static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 1024 /*row statistics*/ + UV_BYTES;
+    static constexpr int TAB_BYTES = 128 * 16 + (BN / 8) * 32 + 128;   // epilogue row and column tables, row -> frame
+    static constexpr int SMEM = RING_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 1024 /*row statistics*/ + UV_BYTES +
+                                TAB_BYTES;
     static constexpr int THREADS = 320;
     static constexpr int EPI_THREADS = 256;
     static constexpr int MAX_S = 4;                            // largest cluster split
@@ -73,6 +75,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * G::STAGES + 1);
     float2 *rowstat = reinterpret_cast<float2 *>(smem + G::RING_BYTES + 256);   // (mean, rstd) of the tile's rows
     float4 *uvs = reinterpret_cast<float4 *>(smem + G::RING_BYTES + 256 + 1024); // (u, v): [frame of the tile][BN]
+    static_assert(sizeof(typename Epi::Row) <= 16 && sizeof(typename Epi::Col) <= 32, "epilogue tables");
+    uint8_t *tab_raw = smem + G::RING_BYTES + 256 + 1024 + G::UV_BYTES;
+    // rows at a stride of 16 bytes from tab_raw, column chunks at a stride of 32 bytes after them
+    uint8_t *rowfr = tab_raw + 128 * 16 + (BN / 8) * 32;     // frame of a tile row, relative to the tile's first frame
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb_all = (K + 63) / 64;
     const int kb0 = (int)((long long)nkb_all * split / S), kb1 = (int)((long long)nkb_all * (split + 1) / S);
@@ -171,15 +177,30 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 if (m < M && n < N) epi.load(m, n, side[i]);
             }
         }
+        if constexpr (Epi::kTables) {
+            // where the rows and the column chunks of this CTA's slice go
+            if (et < rows_per && m0 + r_base + et < M)
+                *reinterpret_cast<typename Epi::Row *>(tab_raw + (r_base + et) * 16) = epi.row_info(m0 + r_base + et);
+            if (et >= 128 && et < 128 + CPR && n0 + (et - 128) * 8 < N)
+                *reinterpret_cast<typename Epi::Col *>(tab_raw + 128 * 16 + (et - 128) * 32) =
+                    epi.col_info(n0 + (et - 128) * 8);
+        }
         if constexpr (Epi::kRowStats) {
             if (epi.ln.on()) {
                 // folded LayerNorm: (u, v) of the tile's columns for every frame the tile's rows belong to, and
                 // (mean, rstd) of the rows this CTA finishes, from the producer's partial sums
                 const int m_last = (m0 + 127 < M ? m0 + 127 : M - 1);
                 const int n_fr = m_last / epi.ln.T - uv_f0 + 1;
+                // layout [frame][pair of columns within a chunk][chunk]: the lanes of a warp, which hold adjacent
+                // chunks, read adjacent 16-byte words
                 for (int idx = et; idx < n_fr * (BN / 2); idx += G::EPI_THREADS) {
                     const int fr = idx / (BN / 2), c2 = idx - fr * (BN / 2);
-                    if (n0 + 2 * c2 < N) uvs[idx] = epi.ln.uv_pair(uv_f0 + fr, n0 + 2 * c2);
+                    if (n0 + 2 * c2 < N)
+                        uvs[(fr * 4 + (c2 & 3)) * CPR + (c2 >> 2)] = epi.ln.uv_pair(uv_f0 + fr, n0 + 2 * c2);
+                }
+                if (et < rows_per) {
+                    const int m = m0 + r_base + et;
+                    rowfr[r_base + et] = (uint8_t)((m < M ? m : M - 1) / epi.ln.T - uv_f0);
                 }
                 // 8 lanes per row, 32 rows per sweep; every load is issued before the first sum
                 constexpr int SWEEPS = 128 / (G::EPI_THREADS / 8);
@@ -299,10 +320,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if constexpr (Epi::kRowStats) {
                         if (epi.ln.on()) {
                             ms = rowstat[tr[i]];
-                            uvp = uvs + ((mm[i] / epi.ln.T - uv_f0) * BN + (nn[i] - n0)) / 2;
+                            uvp = uvs + (int)rowfr[tr[i]] * 4 * CPR + ((nn[i] - n0) >> 3);   // planes CPR words apart
                         }
                     }
-                    epi.apply(mm[i], nn[i], a, side[i], ms, uvp, vmask[i]);
+                    typename Epi::Row rinfo{};
+                    typename Epi::Col cinfo{};
+                    if constexpr (Epi::kTables) {
+                        rinfo = *reinterpret_cast<const typename Epi::Row *>(tab_raw + tr[i] * 16);
+                        cinfo = *reinterpret_cast<const typename Epi::Col *>(tab_raw + 128 * 16 + ((nn[i] - n0) >> 3) * 32);
+                    }
+                    epi.apply(mm[i], nn[i], a, side[i], ms, uvp, CPR, vmask[i], rinfo, cinfo);
                 }
                 if (i0 == 0 && j0 == 0) NFD_TRACE_MARK_T(TRK_OTHER + 7, 64);
             }

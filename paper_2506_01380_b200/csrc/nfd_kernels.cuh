@@ -426,11 +426,13 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float *f) {
 // GEMMs that follow an adaLN turn those partials into (mean, rstd) and apply
 // rstd*(acc - mean*u[n]) + v[n].
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void ln_fold_apply(float *a, const float4 *uv, float2 ms) {
+// uv: (u, v, u, v) of columns 2i, 2i+1 of the item at uv[i * stride]
+__device__ __forceinline__ void ln_fold_apply(float *a, const float4 *uv, int stride, float2 ms) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        a[2 * i] = fmaf(ms.y, fmaf(-ms.x, uv[i].x, a[2 * i]), uv[i].y);
-        a[2 * i + 1] = fmaf(ms.y, fmaf(-ms.x, uv[i].z, a[2 * i + 1]), uv[i].w);
+        const float4 w = uv[i * stride];
+        a[2 * i] = fmaf(ms.y, fmaf(-ms.x, w.x, a[2 * i]), w.y);
+        a[2 * i + 1] = fmaf(ms.y, fmaf(-ms.x, w.z, a[2 * i + 1]), w.w);
     }
 }
 __device__ __forceinline__ void bias_add(float *a, const uint4 &bits) {
@@ -469,13 +471,41 @@ template <typename TS> struct EpiQKV {
     }
     static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
     static constexpr bool kRowStats = true;
+    // Where a row (token) and an 8-column chunk of the output go, worked out once per tile row and tile
+    // column chunk and kept in shared memory, so that an item needs no division.
+    static constexpr bool kTables = true;
+    struct Row {
+        long long q_off;        // m * dh
+        long long kv_off;       // page of the token's frame + tok * dh
+    };
+    struct Col {
+        int which, pad;         // 0 q, 1 k, 2 v
+        long long q_off;        // head * n_rows * dh + e
+        long long kv_off;       // head * T * dh + e
+    };
+    __device__ __forceinline__ Row row_info(int m) const {
+        const int j = m / D.T, tok = m - j * D.T;
+        const FrameDesc &f = sp->fr[j];
+        Row r;
+        r.q_off = (long long)m * D.dh;
+        r.kv_off = (long long)kv_page_offset(D, f.stream, layer, f.frame) + (long long)tok * D.dh;
+        return r;
+    }
+    __device__ __forceinline__ Col col_info(int n) const {
+        Col c;
+        c.which = n / D.d;
+        const int col = n - c.which * D.d;
+        const int head = col / D.dh, e = col - head * D.dh;
+        c.pad = 0;
+        c.q_off = ((long long)head * n_rows) * D.dh + e;
+        c.kv_off = ((long long)head * D.T) * D.dh + e;
+        return c;
+    }
     struct Side {
         uint4 bias;             // unused with the folded LayerNorm (v carries the bias)
         float4 c01, c23;        // (cos, sin) of four adjacent pairs
-        int stream, frame;      // of the token's frame
     };
     __device__ __forceinline__ void load(int m, int n, Side &s) const {
-        const FrameDesc &f = sp->fr[m / D.T];
         if (!ln.on()) s.bias = *reinterpret_cast<const uint4 *>(bias + n);
         const int which = n / D.d, col = n - which * D.d;
         const int e = col % D.dh;
@@ -483,15 +513,12 @@ template <typename TS> struct EpiQKV {
             const float4 *cs = reinterpret_cast<const float4 *>(rope_cs + (size_t)m * (D.dh >> 1) + (e >> 1));
             s.c01 = cs[0], s.c23 = cs[1];
         }
-        s.stream = f.stream, s.frame = f.frame;
     }
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2 ms, const float4 *uv,
-                                          unsigned) const {
-        const int which = n / D.d, col = n - which * D.d;
-        const int head = col / D.dh, e = col - head * D.dh;
-        const int j = m / D.T, tok = m - j * D.T;
+    __device__ __forceinline__ void apply(int, int, float *a, const Side &s, float2 ms, const float4 *uv, int uv_stride,
+                                          unsigned, const Row &row, const Col &col) const {
+        const int which = col.which;
         if (ln.on())
-            ln_fold_apply(a, uv, ms);
+            ln_fold_apply(a, uv, uv_stride, ms);
         else
             bias_add(a, s.bias);
         TS *dst;
@@ -505,12 +532,10 @@ template <typename TS> struct EpiQKV {
                 a[2 * i + 1] = r1;
             }
         }
-        if (which == 0) {
-            dst = q + ((size_t)head * ((size_t)n_rows) + m) * D.dh + e;
-        } else {
-            dst = ((which == 1) ? kc : vc) + kv_page_offset(D, s.stream, layer, s.frame) +
-                  ((size_t)head * D.T + tok) * D.dh + e;
-        }
+        if (which == 0)
+            dst = q + (row.q_off + col.q_off);
+        else
+            dst = ((which == 1) ? kc : vc) + (row.kv_off + col.kv_off);
         *reinterpret_cast<uint4 *>(dst) = pack_bf16x8(a);
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
@@ -558,6 +583,9 @@ template <typename TS> struct EpiGateRes {
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 2;        // epilogue items a thread keeps in flight together
     static constexpr bool kRowStats = false;
+    static constexpr bool kTables = false;
+    struct Row {};
+    struct Col {};
     struct Side {
         uint4 bias;
         float4 g0, g1, z0, z1, s0, s1;
@@ -574,8 +602,8 @@ template <typename TS> struct EpiGateRes {
             s.s0 = sc[0], s.s1 = sc[1];
         }
     }
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2, const float4 *,
-                                          unsigned mask) const {
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2, const float4 *, int,
+                                          unsigned mask, const Row &, const Col &) const {
         float b[8];
         unpack_bf16x8(s.bias, b);
         float4 z0 = s.z0, z1 = s.z1;
@@ -624,6 +652,9 @@ template <typename TS> struct EpiGelu {
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 8;        // epilogue items a thread keeps in flight together
     static constexpr bool kRowStats = true;
+    static constexpr bool kTables = false;
+    struct Row {};
+    struct Col {};
     struct Side {
         uint4 bias;         // unused with the folded LayerNorm (v carries the bias)
     };
@@ -632,9 +663,9 @@ template <typename TS> struct EpiGelu {
         if (!ln.on()) s.bias = *reinterpret_cast<const uint4 *>(bias + n);
     }
     __device__ __forceinline__ void apply(int m, int n, float *a, const Side &s, float2 ms, const float4 *uv,
-                                          unsigned) const {
+                                          int uv_stride, unsigned, const Row &, const Col &) const {
         if (ln.on())
-            ln_fold_apply(a, uv, ms);
+            ln_fold_apply(a, uv, uv_stride, ms);
         else
             bias_add(a, s.bias);
 #pragma unroll
@@ -656,12 +687,15 @@ template <typename TS> struct EpiFinal {
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 4;        // epilogue items a thread keeps in flight together
     static constexpr bool kRowStats = false;
+    static constexpr bool kTables = false;
+    struct Row {};
+    struct Col {};
     struct Side {
         int unused;
     };
     __device__ __forceinline__ void load(int, int, Side &) const {}
-    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &, float2, const float4 *,
-                                          unsigned) const {
+    __device__ __forceinline__ void apply(int m, int n, float *a, const Side &, float2, const float4 *, int,
+                                          unsigned, const Row &, const Col &) const {
 #pragma unroll
         for (int i = 0; i < 8; i += 2) (*this)(m, n + i, a[i], a[i + 1]);
     }
