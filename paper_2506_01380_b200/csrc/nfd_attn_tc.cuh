@@ -367,56 +367,78 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             named_bar_sync(1, 256);
             if (*last_flag) {
                 __threadfence();
-                for (int it = (int)threadIdx.x - 64; it < 128 * 8; it += 256) {
-                    const int r = it >> 3, ch = it & 7;
-                    const int orow = qt * 128 + r;
-                    if (orow >= D.T) continue;
-                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                    float l = 0.f, mx = -INFINITY;
-                    for (int s0 = 0; s0 < nsplit; s0 += 4) {
-                        // four splits at a time, all loads in flight together; this CTA's own state comes from
-                        // shared memory (same values as its published copy)
-                        float2 ml[4];
-                        float4 v0[4], v1[4];
+                // an item = 8 adjacent output columns of a row; two items per thread and round, so that the
+                // loads of both (all splits, four at a time) are in flight together
+                for (int it0 = (int)threadIdx.x - 64; it0 < 128 * 8; it0 += 512) {
+                    int r[2], ch[2];
+                    bool live[2];
+                    float acc[2][8], l[2], mx[2];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int s = s0 + u < nsplit ? s0 + u : nsplit - 1;
-                            if (s == split) {
-                                ml[u] = parkML[r];
-                                const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)r * A::OROW + ch * 8);
-                                v0[u] = po[0], v1[u] = po[1];
-                            } else {
-                                const size_t item = st0 + (size_t)s * 128 + r;
-                                ml[u] = __ldcg(&part_ml[item]);
-                                const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch * 8);
-                                v0[u] = __ldcg(po), v1[u] = __ldcg(po + 1);
+                    for (int q = 0; q < 2; ++q) {
+                        const int it = it0 + q * 256;
+                        r[q] = it >> 3, ch[q] = it & 7;
+                        live[q] = it < 128 * 8 && qt * 128 + r[q] < D.T;
+                        l[q] = 0.f, mx[q] = -INFINITY;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[q][e] = 0.f;
+                    }
+                    for (int s0 = 0; s0 < nsplit; s0 += 4) {
+                        // this CTA's own state comes from shared memory (same values as its published copy)
+                        float2 ml[2][4];
+                        float4 v0[2][4], v1[2][4];
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            if (!live[q]) continue;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int sidx = s0 + u < nsplit ? s0 + u : nsplit - 1;
+                                if (sidx == split) {
+                                    ml[q][u] = parkML[r[q]];
+                                    const float4 *po =
+                                        reinterpret_cast<const float4 *>(parkO + (size_t)r[q] * A::OROW + ch[q] * 8);
+                                    v0[q][u] = po[0], v1[q][u] = po[1];
+                                } else {
+                                    const size_t item = st0 + (size_t)sidx * 128 + r[q];
+                                    ml[q][u] = __ldcg(&part_ml[item]);
+                                    const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch[q] * 8);
+                                    v0[q][u] = __ldcg(po), v1[q][u] = __ldcg(po + 1);
+                                }
                             }
                         }
-                        float mb = mx;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (s0 + u < nsplit) mb = fmaxf(mb, ml[u].x);
-                        const float fo = ex2_approx(mx - mb);          // rescale of what was merged so far (0 at first)
-                        l *= fo;
+                        for (int q = 0; q < 2; ++q) {
+                            if (!live[q]) continue;
+                            float mb = mx[q];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[e] *= fo;
-                        mx = mb;
+                            for (int u = 0; u < 4; ++u)
+                                if (s0 + u < nsplit) mb = fmaxf(mb, ml[q][u].x);
+                            const float fo = ex2_approx(mx[q] - mb);   // rescale of what was merged so far (0 at first)
+                            l[q] *= fo;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (s0 + u < nsplit) {
-                                const float w = ex2_approx(ml[u].x - mx);
-                                l = fmaf(ml[u].y, w, l);
-                                acc[0] = fmaf(v0[u].x, w, acc[0]), acc[1] = fmaf(v0[u].y, w, acc[1]);
-                                acc[2] = fmaf(v0[u].z, w, acc[2]), acc[3] = fmaf(v0[u].w, w, acc[3]);
-                                acc[4] = fmaf(v1[u].x, w, acc[4]), acc[5] = fmaf(v1[u].y, w, acc[5]);
-                                acc[6] = fmaf(v1[u].z, w, acc[6]), acc[7] = fmaf(v1[u].w, w, acc[7]);
+                            for (int e = 0; e < 8; ++e) acc[q][e] *= fo;
+                            mx[q] = mb;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                if (s0 + u < nsplit) {
+                                    const float w = ex2_approx(ml[q][u].x - mb);
+                                    l[q] = fmaf(ml[q][u].y, w, l[q]);
+                                    acc[q][0] = fmaf(v0[q][u].x, w, acc[q][0]), acc[q][1] = fmaf(v0[q][u].y, w, acc[q][1]);
+                                    acc[q][2] = fmaf(v0[q][u].z, w, acc[q][2]), acc[q][3] = fmaf(v0[q][u].w, w, acc[q][3]);
+                                    acc[q][4] = fmaf(v1[q][u].x, w, acc[q][4]), acc[q][5] = fmaf(v1[q][u].y, w, acc[q][5]);
+                                    acc[q][6] = fmaf(v1[q][u].z, w, acc[q][6]), acc[q][7] = fmaf(v1[q][u].w, w, acc[q][7]);
+                                }
                             }
                         }
                     }
-                    const float inv = 1.0f / l;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) acc[u] *= inv;
-                    *reinterpret_cast<uint4 *>(out + (size_t)(j * D.T + orow) * D.d + h * 64 + ch * 8) = pack_bf16x8(acc);
+                    for (int q = 0; q < 2; ++q) {
+                        if (!live[q]) continue;
+                        const float inv = 1.0f / l[q];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) acc[q][u] *= inv;
+                        *reinterpret_cast<uint4 *>(out + (size_t)(j * D.T + qt * 128 + r[q]) * D.d + h * 64 + ch[q] * 8) =
+                            pack_bf16x8(acc[q]);
+                    }
                 }
             }
         }
