@@ -120,6 +120,18 @@ def gelu(x):
     return 0.5 * x * (1.0 + _erf(x / math.sqrt(2.0)))
 
 
+def mlp(h, w1, b1, w2, b2, act: int):
+    """Feed-forward of a block.  act 0: GELU(h W1 + b1) W2 + b2.  act 1: the gated form
+    (SiLU(h Wg + bg) * (h Wu + bu)) W2 + b2, with W1 = [Wg | Wu] side by side; the paper's size table lists an
+    MLP width of about 8/3 of the hidden width for two of its three models, the customary width of this
+    form, and names no activation, so the gated form is offered as a reading, not claimed."""
+    a = h @ w1 + b1
+    if act == 0:
+        return gelu(a) @ w2 + b2
+    dm = w2.shape[0]
+    return (silu(a[:, :dm]) * a[:, dm:]) @ w2 + b2
+
+
 def softmax_rows(s):
     m = np.max(s, axis=-1, keepdims=True)
     e = np.exp(s - m)
@@ -279,7 +291,8 @@ class NFDOracle:
             o = (Pm @ v).transpose(1, 0, 2).reshape(Fn * T, self.d)
             z = z + g1 * (o @ self.w[f"w_o.{l}"] + self.w[f"b_o.{l}"])
             h = self.norm(z) * (1.0 + sc2) + sh2
-            m = gelu(h @ self.w[f"w_fc1.{l}"] + self.w[f"b_fc1.{l}"]) @ self.w[f"w_fc2.{l}"] + self.w[f"b_fc2.{l}"]
+            m = mlp(h, self.w[f"w_fc1.{l}"], self.w[f"b_fc1.{l}"], self.w[f"w_fc2.{l}"], self.w[f"b_fc2.{l}"],
+                    self.cfg.get("act", 0))
             z = z + g2 * m
             if return_aux:
                 aux["K"].append(k)
@@ -332,7 +345,8 @@ class NFDOracle:
                 o[j * T:(j + 1) * T] = (softmax_rows(S) @ Vc).transpose(1, 0, 2).reshape(T, self.d)
             z = z + g1 * (o @ self.w[f"w_o.{l}"] + self.w[f"b_o.{l}"])
             h = self.norm(z) * (1.0 + sc2) + sh2
-            m = gelu(h @ self.w[f"w_fc1.{l}"] + self.w[f"b_fc1.{l}"]) @ self.w[f"w_fc2.{l}"] + self.w[f"b_fc2.{l}"]
+            m = mlp(h, self.w[f"w_fc1.{l}"], self.w[f"b_fc1.{l}"], self.w[f"w_fc2.{l}"], self.w[f"b_fc2.{l}"],
+                    self.cfg.get("act", 0))
             z = z + g2 * m
         if kv_only_last:
             return None, newK, newV

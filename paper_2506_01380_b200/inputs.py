@@ -40,12 +40,19 @@ def make_cfg(name: str, **overrides) -> dict:
     attn      the 16-head x 64 attention shape embedded in a 1-layer model.
     nfd310m   24 layers, d=1024, 16 heads x 64, MLP 4096, 336 tokens/frame, bf16.
     paper130m / paper310m / paper774m: the sizes printed in the paper's appendix
-              table (hidden, MLP, heads, layers).
+              table (hidden, MLP, heads, layers); GELU MLP unless act=1 is passed
+              (gated MLP, the reading that the 8/3 MLP width suggests).
+    tiny_gated / tiny_gated_bf16: the tiny model with a gated MLP of width 340
+              (not a multiple of 8, like the 2730 of the paper's 310M model).
     """
     if name == "tiny":
         cfg = _base_cfg()
     elif name == "tiny_bf16":
         cfg = _base_cfg(dtype=DTYPE_BF16)
+    elif name == "tiny_gated":
+        cfg = _base_cfg(act=1, d_mlp=340)
+    elif name == "tiny_gated_bf16":
+        cfg = _base_cfg(act=1, d_mlp=340, dtype=DTYPE_BF16)
     elif name == "nfd310m":
         cfg = _base_cfg(
             n_layers=24, d_model=1024, n_heads=16, head_dim=64, d_mlp=4096,
@@ -109,8 +116,9 @@ def weight_shapes(cfg) -> dict:
         shapes[f"b_qkv.{l}"] = (3 * d,)
         shapes[f"w_o.{l}"] = (d, d)
         shapes[f"b_o.{l}"] = (d,)
-        shapes[f"w_fc1.{l}"] = (d, dm)
-        shapes[f"b_fc1.{l}"] = (dm,)
+        # act 1 (gated MLP): gate and up projections side by side
+        shapes[f"w_fc1.{l}"] = (d, dm * (2 if cfg.get("act", 0) == 1 else 1))
+        shapes[f"b_fc1.{l}"] = (dm * (2 if cfg.get("act", 0) == 1 else 1),)
         shapes[f"w_fc2.{l}"] = (dm, d)
         shapes[f"b_fc2.{l}"] = (d,)
     return shapes

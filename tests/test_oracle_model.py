@@ -34,9 +34,9 @@ def ctx_inputs(orc, x0, z):
 
 
 # ---------------------------------------------------------------- (1)
-@pytest.mark.parametrize("kind", ["paper", "stress"])
-def test_dense_mask_equals_incremental_cache(kind):
-    cfg = small_cfg()
+@pytest.mark.parametrize("kind,act", [("paper", 0), ("stress", 0), ("stress", 1)])
+def test_dense_mask_equals_incremental_cache(kind, act):
+    cfg = small_cfg(act=act, d_mlp=96 if act == 0 else 100)
     W = cfg["ctx_frames"]
     n_ctx = W + 4                                  # eviction is exercised
     orc = make(cfg, 1, kind)
@@ -212,7 +212,11 @@ def _ref_plain_transformer(cfg, w, X, n_layers):
             o[:, h * dh:(h + 1) * dh] = (e / e.sum(-1, keepdims=True)) @ v[h]
         z = z + o @ w[f"w_o.{l}"] + w[f"b_o.{l}"]
         hmid = ln(z) @ w[f"w_fc1.{l}"] + w[f"b_fc1.{l}"]
-        hmid = np.array([[0.5 * a * (1 + math.erf(a / math.sqrt(2))) for a in row] for row in hmid])
+        if cfg.get("act", 0) == 0:
+            hmid = np.array([[0.5 * a * (1 + math.erf(a / math.sqrt(2))) for a in row] for row in hmid])
+        else:       # gated: columns [0, dm) gate, [dm, 2 dm) up; scalar loops on purpose
+            dm = cfg["d_mlp"]
+            hmid = np.array([[row[i] / (1 + math.exp(-row[i])) * row[dm + i] for i in range(dm)] for row in hmid])
         z = z + hmid @ w[f"w_fc2.{l}"] + w[f"b_fc2.{l}"]
     y = ln(z) @ w["w_out"] + w["b_out"]
     out = np.zeros_like(X)
@@ -224,9 +228,9 @@ def _ref_plain_transformer(cfg, w, X, n_layers):
     return out
 
 
-@pytest.mark.parametrize("patch", [1, 2])
-def test_unmodulated_model_is_a_plain_pre_ln_transformer(patch):
-    cfg = small_cfg(ctx_frames=8, patch=patch)
+@pytest.mark.parametrize("patch,act", [(1, 0), (2, 0), (1, 1)])
+def test_unmodulated_model_is_a_plain_pre_ln_transformer(patch, act):
+    cfg = small_cfg(ctx_frames=8, patch=patch, act=act, d_mlp=96 if act == 0 else 100)
     w = {k: v.astype(np.float64) for k, v in I.make_weights(cfg, 11, "stress").items()}
     d = cfg["d_model"]
     for l in range(cfg["n_layers"]):
@@ -323,6 +327,36 @@ def test_patchify_roundtrip_and_order():
     # token (f=1, row=1, col=0), element (c=2, py=1, px=0)
     assert tok[1 * 4 + 1 * 2 + 0, 2 * 4 + 1 * 2 + 0] == X[1, 2, 1 * 2 + 1, 0 * 2 + 0]
     np.testing.assert_array_equal(orc.unpatchify(tok), X)
+
+
+def test_gated_mlp_special_cases():
+    """The gated feed-forward (act = 1): with the up projection forced to the constant 1 it is a plain SiLU
+    MLP; with the gate pre-activation forced to a large constant it is linear in the up projection
+    (SiLU(c) -> c); shapes are [d, 2 dm] with the gate columns first."""
+    rng = np.random.default_rng(3)
+    d, dm, n = 12, 10, 7
+    h = rng.standard_normal((n, d))
+    w1, b1 = rng.standard_normal((d, 2 * dm)), rng.standard_normal(2 * dm)
+    w2, b2 = rng.standard_normal((dm, d)), rng.standard_normal(d)
+    # general case against scalar loops
+    want = np.zeros((n, d))
+    for r in range(n):
+        a = [sum(h[r, k] * w1[k, c] for k in range(d)) + b1[c] for c in range(2 * dm)]
+        g = [a[i] / (1 + math.exp(-a[i])) * a[dm + i] for i in range(dm)]
+        want[r] = [sum(g[i] * w2[i, o] for i in range(dm)) + b2[o] for o in range(d)]
+    np.testing.assert_allclose(O.mlp(h, w1, b1, w2, b2, 1), want, atol=1e-12)
+    # up == 1: plain SiLU MLP
+    w1u, b1u = w1.copy(), b1.copy()
+    w1u[:, dm:], b1u[dm:] = 0.0, 1.0
+    a = h @ w1[:, :dm] + b1[:dm]
+    np.testing.assert_allclose(O.mlp(h, w1u, b1u, w2, b2, 1), (a / (1 + np.exp(-a))) @ w2 + b2, atol=1e-12)
+    # gate pre-activation == 40: SiLU(40) = 40 to 1e-16, so the block is 40 * (h Wu + bu) W2 + b2
+    w1g, b1g = w1.copy(), b1.copy()
+    w1g[:, :dm], b1g[:dm] = 0.0, 40.0
+    np.testing.assert_allclose(O.mlp(h, w1g, b1g, w2, b2, 1), 40.0 * (h @ w1[:, dm:] + b1[dm:]) @ w2 + b2, rtol=1e-12)
+    # act 0 is untouched by the new branch
+    a0 = h @ w1[:, :dm] + b1[:dm]
+    np.testing.assert_allclose(O.mlp(h, w1[:, :dm], b1[:dm], w2, b2, 0), O.gelu(a0) @ w2 + b2, atol=1e-15)
 
 
 def test_gelu_and_round_bf16():
