@@ -32,6 +32,14 @@ METRIC = "frames/sec at batch 1 (310M-class, 4 steps, k=1)"
 UNIT = "frames/s"
 WORKLOAD = ("nfd310m: 24L d1024 16x64 heads MLP4096 GELU, 336 tokens/frame, 16-frame KV context, "
             "4 steps + commit (commit folded into the next frame's first pass), k=1")
+_STEP = "336 tokens/frame, 16-frame KV context, 4 steps + commit (commit folded into the next frame's first pass), k=1"
+# name -> (inputs.make_cfg name, overrides, description)
+WORKLOADS = {
+    "nfd310m": ("nfd310m", {}, WORKLOAD),
+    "paper130m_gated": ("paper130m", {"act": 1}, "paper130m: 12L d768 12x64 heads gated MLP 2048, " + _STEP),
+    "paper310m_gated": ("paper310m", {"act": 1}, "paper310m: 16L d1024 16x64 heads gated MLP 2730, " + _STEP),
+    "paper774m_gated": ("paper774m", {"act": 1}, "paper774m: 18L d1536 24x64 heads gated MLP 4096, " + _STEP),
+}
 
 
 def peaks():
@@ -111,10 +119,11 @@ def class_work(cfg, T, n_ctx):
 
     def gemm(N, K, res=False):
         return dict(flops=2.0 * M * N * K, bytes=2.0 * (N * K + M * K + M * N) + (8.0 * M * N if res else 0.0))
+    n1 = dm * (2 if cfg.get("act", 0) == 1 else 1)
     return {
         "gemm_qkv_rope_kvstore": gemm(3 * d, d),
         "gemm_out_gate_res": gemm(d, d, True),
-        "gemm_fc1_gelu": gemm(dm, d),
+        "gemm_fc1_gelu": gemm(n1, d),
         "gemm_fc2_gate_res": gemm(d, dm, True),
         "attention": dict(flops=4.0 * M * Nk * d, bytes=2.0 * (2 * Nk * d + 2 * M * d)),
         "adaln_norm": dict(flops=8.0 * M * d, bytes=M * d * 6.0),
@@ -202,7 +211,8 @@ def run_reference(args):
     """Reference arm = the oracle on the host cores (the paper ships no code)."""
     from paper_2506_01380_b200 import inputs as I
     import numpy  # noqa: F401  (loads BLAS so that the thread count is known)
-    cfg = I.make_cfg("nfd310m")
+    wl_cfg, wl_over, wl_text = WORKLOADS[args.workload]
+    cfg = I.make_cfg(wl_cfg, **wl_over)
     steps = max(1, min(args.steps, 6))
     warm = max(0, min(args.warmup, 1))
     times = oracle_sample(cfg, warm + steps)[warm:]
@@ -215,7 +225,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": t_pass * passes_per_frame * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": WORKLOAD},
+            "data": "synthetic", "config": {"workload": wl_text},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -240,6 +250,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the k=4, e2e, profile and CPU legs")
+    ap.add_argument("--workload", default="nfd310m", choices=sorted(WORKLOADS),
+                    help="nfd310m is the configuration the metric is quoted on; the others are the paper's own "
+                         "size-table shapes with a gated MLP (second workload, same step definition)")
     ap.add_argument("--spec-sweep", action="store_true",
                     help="add accepted frames/s for k = 1..4 over action chains of several repeat probabilities")
     args = ap.parse_args()
@@ -262,7 +275,8 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    cfg = I.make_cfg("nfd310m")
+    wl_cfg, wl_over, wl_text = WORKLOADS[args.workload]
+    cfg = I.make_cfg(wl_cfg, **wl_over)
     S, W, T = cfg["n_steps"], cfg["ctx_frames"], I.tokens_per_frame(cfg)
     fs = I.frame_shape(cfg)
     nfd = NFD(cfg, torch_weights(cfg, device, seed=0), device=str(device))
@@ -326,8 +340,9 @@ def main():
     line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": "inputs larger than L2: 604 MB of weights + 528 MB of KV pages are streamed every pass",
+            "config": {"workload": wl_text, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": "inputs larger than L2: the weights (604 MB for nfd310m) and the KV pages (528 MB) are "
+                             "streamed every pass",
                        "forward_passes_of_work_per_step": S + 1, "launched_passes_per_step": S,
                        "cuda_graph": True, "programmatic_dependent_launch": True},
             "clocks": clk, "gpu_launches": int(launches),
@@ -432,11 +447,13 @@ def main():
                 nfd.rollback(1)
             prof = nfd.profile_end()
         roof, shares = roofline_of(cfg, T, W, prof, pk)
+        if roof and args.workload != "nfd310m":
+            roof["traffic"] = None           # the ncu captures are of the nfd310m shape
         line["roofline"] = roof
         line["kernel_time_shares"] = shares
         # whole-pass roofline: the slower of FLOPs at the bf16 peak and bytes at HBM bandwidth
         d, dm, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
-        gemm_params = L * (4 * d * d + 2 * d * dm)
+        gemm_params = L * (4 * d * d + (3 if cfg.get("act", 0) == 1 else 2) * d * dm)
         flops = 2.0 * T * gemm_params + 4.0 * T * (W + 1) * T * d * L
         byts = 2.0 * gemm_params + 2.0 * 2 * L * W * T * d
         t_roof = max(flops / (pk["tf_sust"] * 1e12), byts / (pk["hbm"] * 1e9))

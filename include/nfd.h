@@ -59,7 +59,7 @@ typedef struct {
     int n_streams;                                      /* independent batch slots                               */
     int dtype;                                          /* NFD_DTYPE_*                                           */
     int norm;                                           /* 0 LayerNorm (no affine), 1 RMSNorm                    */
-    int act;                                            /* 0 exact (erf) GELU                                    */
+    int act;                                            /* 0 exact (erf) GELU; 1 gated: SiLU(gate) * up          */
     int rope_t, rope_h, rope_w;                         /* even, sum == head_dim (Section 3.1, 3D pos. emb.)     */
     float rope_theta, norm_eps, t_scale;                /* t_scale multiplies the FM time before the sinusoid    */
     float sigma_d;                                      /* TrigFlow data scale (Section 4.1)                     */
@@ -78,7 +78,7 @@ typedef struct {
     const void *const *w_mod, *const *b_mod; /* [d,6d],[6d]     adaLN: shift,scale,gate (attn), same (mlp) */
     const void *const *w_qkv, *const *b_qkv; /* [d,3d],[3d]     columns: q | k | v, each head-major      */
     const void *const *w_o,   *const *b_o;   /* [d,d],[d]                                                */
-    const void *const *w_fc1, *const *b_fc1; /* [d,d_mlp],[d_mlp]                                        */
+    const void *const *w_fc1, *const *b_fc1; /* [d,d_mlp],[d_mlp]; act 1: [d,2 d_mlp],[2 d_mlp], gate first */
     const void *const *w_fc2, *const *b_fc2; /* [d_mlp,d],[d]                                            */
     const void *w_fmod, *b_fmod;             /* [d,2d],[2d]     final adaLN: shift, scale                */
     const void *w_out, *b_out;               /* [d,P],[P]       velocity head                            */

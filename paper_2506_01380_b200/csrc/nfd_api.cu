@@ -88,7 +88,7 @@ struct nfd_ctx {
     // of the neighbouring GEMMs.  uvtab holds, per cache slot and layer, the (u, v) pairs of the QKV and
     // first MLP projections; ln_stats the row-sum partials of z.
     bool fuse_ln = true;
-    float2 *uvtab = nullptr;                    // [n_slots][L][3d + dm]
+    float2 *uvtab = nullptr;                    // [n_slots][L][3d + n1]
     float2 *ln_stats = nullptr;                 // [Nq_max][d / 32]
     bool fold_active() const {
         const int d = D.d, dm = D.dm;
@@ -140,6 +140,7 @@ static int repack_matrix(nfd_ctx *c, const void *src, int n_in, int n_out, void 
 template <typename TS> static int repack_all(nfd_ctx *c, const nfd_weights *w) {
     const nfd_cfg &g = c->cfg;
     const int d = g.d_model, P = c->D.P, L = g.n_layers, dm = g.d_mlp;
+    const int dmp = c->D.dm, n1 = c->D.n1, act = c->D.act;
     RET(repack_matrix<TS>(c, w->w_pe, P, d, &c->w_pe, true));
     RET(repack_matrix<TS>(c, w->w_pe, P, d, &c->w_pe_io, false));
     RET(repack_matrix<TS>(c, w->b_pe, 1, d, &c->b_pe, false));
@@ -164,9 +165,17 @@ template <typename TS> static int repack_all(nfd_ctx *c, const nfd_weights *w) {
         RET(repack_matrix<TS>(c, w->b_qkv[l], 1, 3 * d, &c->b_qkv[l], false));
         RET(repack_matrix<TS>(c, w->w_o[l], d, d, &c->w_o[l], true));
         RET(repack_matrix<TS>(c, w->b_o[l], 1, d, &c->b_o[l], false));
-        RET(repack_matrix<TS>(c, w->w_fc1[l], d, dm, &c->w_fc1[l], true));
-        RET(repack_matrix<TS>(c, w->b_fc1[l], 1, dm, &c->b_fc1[l], false));
-        RET(repack_matrix<TS>(c, w->w_fc2[l], dm, d, &c->w_fc2[l], true));
+        // MLP: hidden width padded to dmp with zero weights; gate and up columns of the gated form interleaved
+        if (!w->w_fc1[l] || !w->b_fc1[l] || !w->w_fc2[l]) return NFD_E_NULLPTR;
+        RET(dev_alloc(c, &c->w_fc1[l], (size_t)n1 * d * sizeof(TS)));
+        RET(dev_alloc(c, &c->b_fc1[l], (size_t)n1 * sizeof(TS)));
+        RET(dev_alloc(c, &c->w_fc2[l], (size_t)d * dmp * sizeof(TS)));
+        k_repack_fc1<TS><<<(unsigned)(((size_t)n1 * d + 255) / 256), 256, 0, c->st>>>((const TS *)w->w_fc1[l],
+                                                                                      (TS *)c->w_fc1[l], d, dm, dmp, act);
+        k_repack_fc1<TS><<<(n1 + 255) / 256, 256, 0, c->st>>>((const TS *)w->b_fc1[l], (TS *)c->b_fc1[l], 1, dm, dmp, act);
+        k_repack_fc2<TS><<<(unsigned)(((size_t)d * dmp + 255) / 256), 256, 0, c->st>>>((const TS *)w->w_fc2[l],
+                                                                                       (TS *)c->w_fc2[l], d, dm, dmp);
+        CK(cudaGetLastError());
         RET(repack_matrix<TS>(c, w->b_fc2[l], 1, d, &c->b_fc2[l], false));
     }
     return NFD_OK;
@@ -194,7 +203,7 @@ static int validate_cfg(const nfd_cfg &g) {
     if (g.n_streams < 1 || g.n_streams > 1024) return NFD_E_BADCFG;
     if (g.dtype != NFD_DTYPE_FP32 && g.dtype != NFD_DTYPE_BF16) return NFD_E_BADCFG;
     if (g.norm != 0 && g.norm != 1) return NFD_E_BADCFG;
-    if (g.act != 0) return NFD_E_BADCFG;
+    if (g.act != 0 && g.act != 1) return NFD_E_BADCFG;
     if (g.rope_t < 0 || g.rope_h < 0 || g.rope_w < 0 || (g.rope_t | g.rope_h | g.rope_w) & 1) return NFD_E_BADCFG;
     if (g.rope_t + g.rope_h + g.rope_w != g.head_dim) return NFD_E_BADCFG;
     if (!(g.rope_theta > 0.f) || !(g.norm_eps > 0.f) || !(g.sigma_d > 0.f)) return NFD_E_BADCFG;
@@ -308,7 +317,7 @@ template <typename TS> static void enqueue_conditioning(nfd_ctx *c, int rows) {
     const int d = D.d, L = D.L, nf = rows;
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
-    const size_t uv_row = (size_t)L * (3 * d + D.dm);
+    const size_t uv_row = (size_t)L * (3 * d + D.n1);
     const bool fold = c->fold_active();
     c->cls = CLS_COND;
     {
@@ -326,9 +335,9 @@ template <typename TS> static void enqueue_conditioning(nfd_ctx *c, int rows) {
                 (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, (const float *)c->sc, c->fmod, d, 2 * d,
                 (size_t)2 * d, (size_t)0);
         if (fold)
-            PLAUNCH(c, (k_modw<TS>), dim3((3 * d + D.dm + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wqkv,
+            PLAUNCH(c, (k_modw<TS>), dim3((3 * d + D.n1 + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wqkv,
                     (const TS *const *)c->dp_bqkv, (const TS *const *)c->dp_wfc1, (const TS *const *)c->dp_bfc1,
-                    (const float *)c->mod, mod_row, c->uvtab, uv_row, d, D.dm);
+                    (const float *)c->mod, mod_row, c->uvtab, uv_row, d, D.n1);
     }
 }
 
@@ -338,7 +347,7 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     const int d = D.d, L = D.L, M = nf * D.T;
     const StepParams *sp = c->d_sp;
     const size_t mod_row = (size_t)L * 6 * d;
-    const size_t uv_row = (size_t)L * (3 * d + D.dm);
+    const size_t uv_row = (size_t)L * (3 * d + D.n1);
     const bool fold = c->fold_active();
     // conditioning: only for the (t, action) pairs that are not in the modulation cache
     if (c->h_sp.nc > 0) enqueue_conditioning<TS>(c, nf);
@@ -355,7 +364,7 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
         // with the folded LayerNorm hbuf already holds z*(1+scale) and ln_stats the row sums of z
         LnFold lq{nullptr, uv_row, c->ln_stats, d / 32, D.norm, D.eps, sp, D.T}, lm = lq;
         if (fold) {
-            lq.uv = c->uvtab + (size_t)l * (3 * d + D.dm);
+            lq.uv = c->uvtab + (size_t)l * (3 * d + D.n1);
             lm.uv = lq.uv + 3 * d;
         } else {
             c->cls = CLS_ADALN;
@@ -373,15 +382,15 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
                           fold ? (TS *)c->hbuf : (TS *)nullptr, modl + 4 * d, fold ? c->ln_stats : (float2 *)nullptr};
         c->cls = CLS_GEMM_O;
         launch_gemm<TS>(c, (const TS *)c->abuf, (const TS *)c->w_o[l], M, d, d, eo, TC_RES, c->w_fc1[l],
-                        (size_t)d * D.dm, fold);
+                        (size_t)d * D.n1, fold);
         if (!fold) {
             c->cls = CLS_ADALN;
             PLAUNCH(c, (k_adaln<TS>), ln_grid, 128, 0, sp, D, (const float *)c->z, (TS *)c->hbuf, modl, mod_row,
                     (size_t)3 * d, (size_t)4 * d);
         }
-        EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.dm, lm};
+        EpiGelu<TS> eg{(const TS *)c->b_fc1[l], (TS *)c->mbuf, D.n1, D.act, lm};
         c->cls = CLS_GEMM_FC1;
-        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.dm, d, eg, TC_GELU, c->w_fc2[l],
+        launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_fc1[l], M, D.n1, d, eg, TC_GELU, c->w_fc2[l],
                         (size_t)d * D.dm, fold);
         // the last layer's output goes to the final adaLN kernel, which reads z itself
         const bool more = fold && l + 1 < L;
@@ -618,7 +627,8 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     c->bf16_mode = cfg->dtype == NFD_DTYPE_BF16;
     c->esz = c->bf16_mode ? 2 : 4;
     Dims &D = c->D;
-    D.L = cfg->n_layers, D.d = cfg->d_model, D.H = cfg->n_heads, D.dh = cfg->head_dim, D.dm = cfg->d_mlp;
+    D.L = cfg->n_layers, D.d = cfg->d_model, D.H = cfg->n_heads, D.dh = cfg->head_dim;
+    D.dm = (cfg->d_mlp + 7) / 8 * 8, D.act = cfg->act, D.n1 = D.act ? 2 * D.dm : D.dm;
     D.C = cfg->latent_c, D.Hl = cfg->latent_h, D.Wl = cfg->latent_w, D.p = cfg->patch;
     D.th = D.Hl / D.p, D.tw = D.Wl / D.p, D.T = D.th * D.tw, D.P = D.C * D.p * D.p;
     // ring pages per layer: the window, the frames of a speculation and the deferred frames that may ride along
@@ -653,7 +663,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     A((void **)&c->mod, (size_t)n_slots * D.L * 6 * D.d * 4);
     A((void **)&c->fmod, (size_t)n_slots * 2 * D.d * 4);
     if (c->bf16_mode) {
-        A((void **)&c->uvtab, (size_t)n_slots * D.L * (3 * D.d + D.dm) * sizeof(float2));
+        A((void **)&c->uvtab, (size_t)n_slots * D.L * (3 * D.d + D.n1) * sizeof(float2));
         A((void **)&c->ln_stats, Mmax * ((D.d + 31) / 32) * sizeof(float2));
     }
     A((void **)&c->pend_x0, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);

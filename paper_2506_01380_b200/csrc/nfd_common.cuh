@@ -48,7 +48,10 @@ struct StepParams {
 
 // Static model dimensions, passed by value to kernels.
 struct Dims {
-    int L, d, H, dh, dm;
+    int L, d, H, dh;
+    int dm;                 // MLP width as stored: the configured width rounded up to a multiple of 8
+    int n1;                 // output columns of the first MLP projection: dm, or 2*dm for the gated form
+    int act;                // 0 GELU, 1 gated (SiLU(gate) * up; gate and up columns interleaved)
     int C, Hl, Wl, p, th, tw, T, P;
     int R, W, n_streams;
     int norm;
@@ -150,6 +153,8 @@ __device__ __forceinline__ size_t kv_page_offset(const Dims &D, int stream, int 
 }
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+// for values that are rounded to bf16 afterwards
+__device__ __forceinline__ float silu_fast_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
 
 // GELU (erf form) for values that are rounded to bf16 afterwards: erf by the

@@ -647,7 +647,8 @@ template <typename TS> struct EpiGateRes {
 template <typename TS> struct EpiGelu {
     const TS *bias;
     TS *out;
-    int N;
+    int N;                  // columns of the GEMM (n1)
+    int act;                // 0: out[m][n] = GELU(.); 1: out[m][n/2] = SiLU(gate) * up, (gate, up) = columns (n, n+1)
     LnFold ln;              // folded adaLN in front of this projection (tensor-core path only)
     __device__ __forceinline__ void prefetch(unsigned int, unsigned int) const {}
     static constexpr int kBatch = 8;        // epilogue items a thread keeps in flight together
@@ -668,11 +669,23 @@ template <typename TS> struct EpiGelu {
             ln_fold_apply(a, uv, uv_stride, ms);
         else
             bias_add(a, s.bias);
+        if (act == 0) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i]);
-        *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
+            for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i]);
+            *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
+        } else {
+            uint2 o;
+            __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&o);
+            h[0] = __floats2bfloat162_rn(silu_fast_f(a[0]) * a[1], silu_fast_f(a[2]) * a[3]);
+            h[1] = __floats2bfloat162_rn(silu_fast_f(a[4]) * a[5], silu_fast_f(a[6]) * a[7]);
+            *reinterpret_cast<uint2 *>(out + (size_t)m * (N >> 1) + (n >> 1)) = o;
+        }
     }
     __device__ __forceinline__ void operator()(int m, int n, float a0, float a1) const {
+        if (act) {
+            out[(size_t)m * (N >> 1) + (n >> 1)] = from_f<TS>(silu_f(a0 + to_f(bias[n])) * (a1 + to_f(bias[n + 1])));
+            return;
+        }
         TS *o = out + (size_t)m * N + n;
         o[0] = from_f<TS>(gelu_erf_f(a0 + to_f(bias[n])));
         o[1] = from_f<TS>(gelu_erf_f(a1 + to_f(bias[n + 1])));
@@ -905,6 +918,29 @@ __global__ void k_kv_hash(Dims D, const TS *kc, const TS *vc, int stream, int fi
 }
 
 // transpose [rows][cols] -> [cols][rows]
+// First MLP projection, repacked as [n1][d] (one row per output column): row r is column r of the caller's
+// [d][dm] matrix (act 0) or, for the gated form ([d][2 dm], gate columns first), rows 2i and 2i+1 are the gate
+// and the up column of hidden unit i, so that a GEMM epilogue finds both in adjacent accumulators.  Rows of
+// the padding (hidden units dm .. dmp-1) are zero.  n_in = 1 repacks the bias the same way.
+template <typename TS>
+__global__ void k_repack_fc1(const TS *src, TS *dst, int n_in, int dm, int dmp, int act) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int n1 = act ? 2 * dmp : dmp;
+    if (idx >= (size_t)n1 * n_in) return;
+    const int r = (int)(idx / n_in), i = (int)(idx % n_in);
+    const int unit = act ? r >> 1 : r;
+    const int col = act ? ((r & 1) ? dm + unit : unit) : r;
+    dst[idx] = unit < dm ? src[(size_t)i * (act ? 2 * dm : dm) + col] : from_f<TS>(0.f);
+}
+// Second MLP projection, repacked as [d][dmp] with zero columns for the padding.
+template <typename TS>
+__global__ void k_repack_fc2(const TS *src, TS *dst, int d, int dm, int dmp) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)d * dmp) return;
+    const int o = (int)(idx / dmp), k = (int)(idx % dmp);
+    dst[idx] = k < dm ? src[(size_t)k * d + o] : from_f<TS>(0.f);
+}
+
 template <typename TS>
 __global__ void k_transpose(const TS *in, TS *out, int rows, int cols) {
     __shared__ TS tile[32][33];

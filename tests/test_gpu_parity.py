@@ -77,6 +77,11 @@ CASES = [
     ("tiny_bf16", "stress", {}),
     ("tiny_bf16", "paper", {"fuse_ln": 0}),       # in-layer adaLN as kernels of their own
     ("tiny_bf16", "stress", {"fuse_ln": 0}),
+    ("tiny_gated", "stress", {}),                 # gated MLP of width 340 (padded to 344 inside)
+    ("tiny_gated_bf16", "paper", {}),
+    ("tiny_gated_bf16", "stress", {}),
+    ("tiny_gated_bf16", "stress", {"fuse_ln": 0}),
+    ("tiny_gated_bf16", "stress", {"fast": 0}),
 ]
 
 
@@ -274,6 +279,19 @@ def test_310m_slice_two_layers(kind, fuse_ln):
     """Two layers at model width, with the in-layer LayerNorms folded into the neighbouring GEMMs (the
     default) and as kernels of their own."""
     _teacher_forced(I.make_cfg("nfd310m_slice"), kind, n_prompt=5, k=2, seed=0, fuse_ln=fuse_ln)
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_paper_310m_shape_two_layers(act):
+    """The paper's own 310M row of its size table (hidden 1024, MLP 2730, 16 heads), two layers of it: an
+    MLP width that is no multiple of 8, as GELU MLP and as gated MLP."""
+    _teacher_forced(I.make_cfg("paper310m", n_layers=2, act=act), "stress", n_prompt=3, k=2, seed=act)
+
+
+def test_paper_130m_and_774m_shapes_one_layer():
+    """Hidden widths 768 (12 heads) and 1536 (24 heads) of the paper's size table, gated MLP."""
+    for name in ("paper130m", "paper774m"):
+        _teacher_forced(I.make_cfg(name, n_layers=1, act=1, ctx_frames=2), "paper", n_prompt=2, k=1, seed=3)
 
 
 def test_310m_full_config_teacher_forced():
