@@ -138,40 +138,57 @@ template <typename TS>
 __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *const *Wqkv_l, const TS *const *bqkv_l,
                                               const TS *const *Wfc1_l, const TS *const *bfc1_l, const float *mod,
                                               size_t mod_row_stride, float2 *uv, size_t uv_row_stride, int d, int dm) {
+    // (1 + scale) and shift of up to four conditioning rows, 1024 columns at a time: every warp of the CTA
+    // works on the same layer and projection, so they are fetched once per CTA
+    __shared__ __align__(16) float s_sc[4][1024];
+    __shared__ __align__(16) float s_sh[4][1024];
     NFD_TRACE_T0();
     pdl_wait();
     pdl_launch();
     constexpr int NV = WVec<TS>::N;
     const int layer = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int o = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (o >= 3 * d + dm) return;
-    const bool mlp = o >= 3 * d;
+    const int o_cta = blockIdx.x * (blockDim.x >> 5);          // 3d is a multiple of the 8 outputs of a CTA
+    const int o = o_cta + warp;
+    const bool live = o < 3 * d + dm;
+    const bool mlp = o_cta >= 3 * d;
     const int oo = mlp ? o - 3 * d : o;
-    const TS *wrow = (mlp ? Wfc1_l[layer] : Wqkv_l[layer]) + (size_t)oo * d;
-    const float bo = to_f((mlp ? bfc1_l[layer] : bqkv_l[layer])[oo]);
+    const TS *wrow = (mlp ? Wfc1_l[layer] : Wqkv_l[layer]) + (size_t)(live ? oo : 0) * d;
+    const float bo = live ? to_f((mlp ? bfc1_l[layer] : bqkv_l[layer])[oo]) : 0.f;
     const size_t off_shift = (size_t)layer * 6 * d + (mlp ? 3 * d : 0);
     const size_t off_scale = off_shift + d;
     const int nc = sp->nc;
     for (int c0 = 0; c0 < nc; c0 += 4) {
         float au[4] = {0.f, 0.f, 0.f, 0.f}, av[4] = {0.f, 0.f, 0.f, 0.f};
-        const float *mrow[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) mrow[r] = mod + (size_t)sp->cd[c0 + r < nc ? c0 + r : c0].slot * mod_row_stride;
-        for (int i = lane * NV; i < d; i += 32 * NV) {
-            float w[NV];
-            WVec<TS>::load(wrow + i, w);
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
+        for (int i0 = 0; i0 < d; i0 += 1024) {
+            const int span = d - i0 < 1024 ? d - i0 : 1024;
+            __syncthreads();
+            for (int idx = threadIdx.x * 4; idx < 4 * span; idx += blockDim.x * 4) {
+                const int r = idx / span, i = idx - r * span;
                 if (c0 + r < nc) {
+                    const float *mrow = mod + (size_t)sp->cd[c0 + r].slot * mod_row_stride;
+                    const float4 sc = *reinterpret_cast<const float4 *>(mrow + off_scale + i0 + i);
+                    *reinterpret_cast<float4 *>(&s_sc[r][i]) = make_float4(1.0f + sc.x, 1.0f + sc.y, 1.0f + sc.z, 1.0f + sc.w);
+                    *reinterpret_cast<float4 *>(&s_sh[r][i]) = *reinterpret_cast<const float4 *>(mrow + off_shift + i0 + i);
+                }
+            }
+            __syncthreads();
+            if (!live) continue;
+            for (int i = lane * NV; i < span; i += 32 * NV) {
+                float w[NV];
+                WVec<TS>::load(wrow + i0 + i, w);
 #pragma unroll
-                    for (int e = 0; e < NV; e += 4) {
-                        const float4 sc = *reinterpret_cast<const float4 *>(mrow[r] + off_scale + i + e);
-                        const float4 sh = *reinterpret_cast<const float4 *>(mrow[r] + off_shift + i + e);
-                        au[r] = fmaf(w[e], 1.0f + sc.x, au[r]), av[r] = fmaf(w[e], sh.x, av[r]);
-                        au[r] = fmaf(w[e + 1], 1.0f + sc.y, au[r]), av[r] = fmaf(w[e + 1], sh.y, av[r]);
-                        au[r] = fmaf(w[e + 2], 1.0f + sc.z, au[r]), av[r] = fmaf(w[e + 2], sh.z, av[r]);
-                        au[r] = fmaf(w[e + 3], 1.0f + sc.w, au[r]), av[r] = fmaf(w[e + 3], sh.w, av[r]);
+                for (int r = 0; r < 4; ++r) {
+                    if (c0 + r < nc) {
+#pragma unroll
+                        for (int e = 0; e < NV; e += 4) {
+                            const float4 sc = *reinterpret_cast<const float4 *>(&s_sc[r][i + e]);
+                            const float4 sh = *reinterpret_cast<const float4 *>(&s_sh[r][i + e]);
+                            au[r] = fmaf(w[e], sc.x, au[r]), av[r] = fmaf(w[e], sh.x, av[r]);
+                            au[r] = fmaf(w[e + 1], sc.y, au[r]), av[r] = fmaf(w[e + 1], sh.y, av[r]);
+                            au[r] = fmaf(w[e + 2], sc.z, au[r]), av[r] = fmaf(w[e + 2], sh.z, av[r]);
+                            au[r] = fmaf(w[e + 3], sc.w, au[r]), av[r] = fmaf(w[e + 3], sh.w, av[r]);
+                        }
                     }
                 }
             }
@@ -180,7 +197,7 @@ __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *co
         for (int r = 0; r < 4; ++r) {
             if (c0 + r >= nc) break;
             const float su = warp_sum(au[r]), sv = warp_sum(av[r]);
-            if (lane == 0)
+            if (lane == 0 && live)
                 uv[(size_t)sp->cd[c0 + r].slot * uv_row_stride + (size_t)layer * (3 * d + dm) + o] =
                     make_float2(su, sv + bo);
         }
