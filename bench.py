@@ -260,6 +260,8 @@ def main():
     ap.add_argument("--workload", default="nfd310m", choices=sorted(WORKLOADS),
                     help="nfd310m is the configuration the metric is quoted on; the others are the paper's own "
                          "size-table shapes with a gated MLP (second workload, same step definition)")
+    ap.add_argument("--batch8", action="store_true",
+                    help="add the 8-stream, 32-frame-context leg (aggregate and per-stream frames/s)")
     ap.add_argument("--spec-sweep", action="store_true",
                     help="add accepted frames/s for k = 1..4 over action chains of several repeat probabilities")
     args = ap.parse_args()
@@ -416,6 +418,45 @@ def main():
         line["spec_k4"] = {"accepted_frames_per_s": round(acc / (ms4 * 1e-3), 3), "acceptance_rate": round(acc / spec, 4),
                            "accepted_per_pass": round(acc / passes, 4), "ms_per_speculate": round(ms4 / passes, 4),
                            "p_repeat": 0.8, "frames": acc}
+
+        # ---------------- 8 independent streams, 32-frame context, one batched call per frame ----------------
+        if args.batch8:
+            nb = 8
+            cfg8 = dict(cfg, ctx_frames=32, n_streams=nb)
+            nfd.close()
+            nfd8 = NFD(cfg8, torch_weights(cfg8, device, seed=0), device=str(device))
+            nfd8.warm_modulation()
+            streams = list(range(nb))
+            for st in streams:
+                acts = I.make_actions_uniform(cfg8, 32, 100 + st)
+                for i in range(0, 32, 4):
+                    nfd8.commit_frame(randn(4, *fs), acts[i:i + 4], randn(4, *fs), stream=st)
+            n8 = 16
+            acts8 = [I.make_actions_uniform(cfg8, n8 + 3, st) for st in streams]
+            nz8, cz8 = randn(S, nb, 1, *fs), randn(nb, 1, *fs)
+            x8 = torch.empty((nb, 1) + fs, device=device)
+            with torch.cuda.stream(nfd8.stream):
+                for i in range(3):
+                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
+                    for st in streams:
+                        nfd8.rollback(1, stream=st)
+                torch.cuda.synchronize(device)
+                e0.record(nfd8.stream)
+                for i in range(3, n8 + 3):
+                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
+                    for st in streams:
+                        nfd8.rollback(1, stream=st)
+                e1.record(nfd8.stream)
+                torch.cuda.synchronize(device)
+            assert nfd8.status() == 0
+            ms8 = e0.elapsed_time(e1)
+            line["batch8_ctx32"] = {"aggregate_frames_per_s": round(nb * n8 / (ms8 * 1e-3), 2),
+                                    "per_stream_frames_per_s": round(n8 / (ms8 * 1e-3), 2),
+                                    "ms_per_batched_frame_step": round(ms8 / n8, 3), "streams": nb, "ctx_frames": 32,
+                                    "steps": n8}
+            nfd8.close()
+            nfd = NFD(cfg, torch_weights(cfg, device, seed=0), device=str(device))
+            nfd.warm_modulation()
 
         # ---------------- speculation depth x action repeat probability ----------------
         if args.spec_sweep:

@@ -58,9 +58,12 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
         pl.KB = KB;
         pl.BPF = D.T / KB;
         pl.QT = (D.T + 127) / 128;
-        // split the longest window (a frame sees at most W + 1 pages) so that heads x query tiles x splits
-        // fills the SMs once
-        const int target = fs.n_sm / (D.H * pl.QT) > 1 ? fs.n_sm / (D.H * pl.QT) : 1;
+        // split the longest window (a frame sees at most W + 1 pages) so that streams x heads x query tiles x
+        // splits fills the SMs once: a context made for several streams is run with batched passes, which bring
+        // enough (frame, head, query tile) items by themselves, and long unsplit key ranges amortise the
+        // start and the merge of a CTA.  The split depends on the configuration only, never on the pass.
+        const int items_per_pass = D.n_streams * D.H * pl.QT;
+        const int target = fs.n_sm / items_per_pass > 1 ? fs.n_sm / items_per_pass : 1;
         pl.CH = ((D.W + 1) * pl.BPF + target - 1) / target;
         pl.MAXSPLIT = ((D.W + 1) * pl.BPF + pl.CH - 1) / pl.CH;
         if (pl.MAXSPLIT > 1) {
@@ -203,12 +206,12 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
     return best;
 }
 
-template <int BN, typename Epi>
-static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const bf16 *A, const bf16 *Wt, int M, int N, int K, int S,
-                           Epi epi, L2Prefetch pf) {
+template <int BN, typename Epi, int SC>
+static bool launch_gemm_tc_sc(FastState &fs, cudaStream_t st, const bf16 *A, const bf16 *Wt, int M, int N, int K, int S,
+                              Epi epi, L2Prefetch pf) {
     using G = GemmCfg<BN>;
     static bool attr_set = false;
-    auto kern = k_gemm_tc<BN, Epi>;
+    auto kern = k_gemm_tc<BN, Epi, SC>;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM) != cudaSuccess) {
             cudaGetLastError();
@@ -228,6 +231,14 @@ static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const bf16 *A, const 
         return false;
     }
     return true;
+}
+
+// the unsplit case has a kernel of its own (see k_gemm_tc)
+template <int BN, typename Epi>
+static bool launch_gemm_tc(FastState &fs, cudaStream_t st, const bf16 *A, const bf16 *Wt, int M, int N, int K, int S,
+                           Epi epi, L2Prefetch pf) {
+    if (S == 1) return launch_gemm_tc_sc<BN, Epi, 1>(fs, st, A, Wt, M, N, K, S, epi, pf);
+    return launch_gemm_tc_sc<BN, Epi, 0>(fs, st, A, Wt, M, N, K, S, epi, pf);
 }
 
 template <typename TS, typename Epi>

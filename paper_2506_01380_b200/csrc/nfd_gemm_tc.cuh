@@ -55,11 +55,16 @@ struct L2Prefetch {
     unsigned long long bytes;      // multiple of 16; 0 = nothing
 };
 
-template <int BN, typename Epi>
+// SC: the split factor when it is known at compile time (1: no cluster; the epilogue then works on four items at
+// a time instead of two, which gives its dependent instruction chains more to overlap with), 0: run-time S.
+template <int BN, typename Epi, int SC = 0>
 __global__ void __launch_bounds__(GemmCfg<BN>::THREADS, GemmCfg<BN>::MIN_CTAS)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int M, int N, int K,
-          int S, Epi epi, L2Prefetch pf, int *status) {
+          int S_rt, Epi epi, L2Prefetch pf, int *status) {
     using G = GemmCfg<BN>;
+    const int S = SC ? SC : S_rt;
+    constexpr int GRP = SC == 1 ? 4 : 2;                     // epilogue items finished together
+    constexpr int NS = SC == 1 ? 1 : G::MAX_S;               // partials kept per item
     constexpr int MAX_ITEMS = Epi::kBatch;                   // epilogue items in flight together per thread
     extern __shared__ uint8_t smem_raw[];
     NFD_TRACE_T0();
@@ -282,10 +287,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 vmask[i] = __ballot_sync(0xffffffffu, mm[i] >= 0);
             }
 #pragma unroll
-            for (int j0 = 0; j0 < MAX_ITEMS; j0 += 2) {
-                float4 u0[2][G::MAX_S], u1[2][G::MAX_S];
+            for (int j0 = 0; j0 < MAX_ITEMS; j0 += GRP) {
+                float4 u0[GRP][NS], u1[GRP][NS];
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
+                for (int jj = 0; jj < GRP; ++jj) {
                     const int i = j0 + jj;
                     if (i >= MAX_ITEMS || mm[i] < 0) continue;
                     const uint32_t off = (uint32_t)(tr[i] * G::SROW + (nn[i] - n0)) * 4;
@@ -294,7 +299,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                         u0[jj][0] = *reinterpret_cast<const float4 *>(p), u1[jj][0] = *reinterpret_cast<const float4 *>(p + 4);
                     } else {
 #pragma unroll
-                        for (int sp_ = 0; sp_ < G::MAX_S; ++sp_) {
+                        for (int sp_ = 0; sp_ < NS; ++sp_) {
                             if (sp_ < S) {
                                 const uint32_t ra = cluster_map(stage_u32 + off, (uint32_t)sp_);
                                 u0[jj][sp_] = ld_cluster_f4(ra), u1[jj][sp_] = ld_cluster_f4(ra + 16);
@@ -303,12 +308,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     }
                 }
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
+                for (int jj = 0; jj < GRP; ++jj) {
                     const int i = j0 + jj;
                     if (i >= MAX_ITEMS || mm[i] < 0) continue;
                     float4 v0 = u0[jj][0], v1 = u1[jj][0];
 #pragma unroll
-                    for (int sp_ = 1; sp_ < G::MAX_S; ++sp_) {
+                    for (int sp_ = 1; sp_ < NS; ++sp_) {
                         if (sp_ < S) {
                             v0.x += u0[jj][sp_].x, v0.y += u0[jj][sp_].y, v0.z += u0[jj][sp_].z, v0.w += u0[jj][sp_].w;
                             v1.x += u1[jj][sp_].x, v1.y += u1[jj][sp_].y, v1.z += u1[jj][sp_].z, v1.w += u1[jj][sp_].w;
