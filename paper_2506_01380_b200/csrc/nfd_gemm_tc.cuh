@@ -31,7 +31,9 @@
 #include "nfd_sm100.cuh"
 
 template <int BN> struct GemmCfg {
-    static constexpr int STAGES = BN <= 32 ? 7 : 6;             // ring deep enough that one CTA owns an SM
+    // ring deep enough that one CTA owns an SM; the wide tiles (passes of several frames) keep about the same
+    // number of bytes in flight with fewer, larger stages
+    static constexpr int STAGES = BN <= 32 ? 7 : (BN <= 128 ? 6 : (BN <= 192 ? 4 : 3));
     static constexpr int A_BYTES = 128 * 128;                  // 128 rows x 64 bf16
     static constexpr int B_BYTES = BN * 128;
     static constexpr int RING_BYTES = STAGES * (A_BYTES + B_BYTES);
