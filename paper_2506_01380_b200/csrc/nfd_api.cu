@@ -335,7 +335,7 @@ template <typename TS> static void enqueue_conditioning(nfd_ctx *c, int rows) {
                 (const TS *const *)(c->dp_fmod + 1), (const TS *)nullptr, (const float *)c->sc, c->fmod, d, 2 * d,
                 (size_t)2 * d, (size_t)0);
         if (fold)
-            PLAUNCH(c, (k_modw<TS>), dim3((3 * d + D.n1 + 7) / 8, L), 256, 0, sp, (const TS *const *)c->dp_wqkv,
+            PLAUNCH(c, (k_modw<TS>), dim3((3 * d + D.n1 + MODW_OUT - 1) / MODW_OUT, L), 256, 0, sp, (const TS *const *)c->dp_wqkv,
                     (const TS *const *)c->dp_bqkv, (const TS *const *)c->dp_wfc1, (const TS *const *)c->dp_bfc1,
                     (const float *)c->mod, mod_row, c->uvtab, uv_row, d, D.n1);
     }

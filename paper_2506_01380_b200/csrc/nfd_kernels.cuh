@@ -131,9 +131,10 @@ __global__ void __launch_bounds__(256) k_gemv(const StepParams *sp, const TS *co
 // and apply mean and rstd per row in its epilogue.  u and v depend on the
 // conditioning row only and are kept in the modulation cache next to shift and
 // scale.  This kernel fills (u, v) for the QKV projection (outputs 0..3d) and
-// the first MLP projection (outputs 3d..3d+dm) of layer blockIdx.y, one warp
-// per output, four conditioning rows at a time.
+// the first MLP projection (outputs 3d..3d+dm) of layer blockIdx.y: 64 outputs
+// per CTA (one warp per output, eight in turn), four conditioning rows at a time.
 // ---------------------------------------------------------------------------
+#define MODW_OUT 64          // outputs per CTA of k_modw (8 per warp)
 template <typename TS>
 __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *const *Wqkv_l, const TS *const *bqkv_l,
                                               const TS *const *Wfc1_l, const TS *const *bfc1_l, const float *mod,
@@ -148,18 +149,14 @@ __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *co
     constexpr int NV = WVec<TS>::N;
     const int layer = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int o_cta = blockIdx.x * (blockDim.x >> 5);          // 3d is a multiple of the 8 outputs of a CTA
-    const int o = o_cta + warp;
-    const bool live = o < 3 * d + dm;
+    const int o_cta = blockIdx.x * MODW_OUT;                   // 3d is a multiple of the outputs of a CTA
     const bool mlp = o_cta >= 3 * d;
-    const int oo = mlp ? o - 3 * d : o;
-    const TS *wrow = (mlp ? Wfc1_l[layer] : Wqkv_l[layer]) + (size_t)(live ? oo : 0) * d;
-    const float bo = live ? to_f((mlp ? bfc1_l[layer] : bqkv_l[layer])[oo]) : 0.f;
+    const TS *W = mlp ? Wfc1_l[layer] : Wqkv_l[layer];
+    const TS *B = mlp ? bfc1_l[layer] : bqkv_l[layer];
     const size_t off_shift = (size_t)layer * 6 * d + (mlp ? 3 * d : 0);
     const size_t off_scale = off_shift + d;
     const int nc = sp->nc;
     for (int c0 = 0; c0 < nc; c0 += 4) {
-        float au[4] = {0.f, 0.f, 0.f, 0.f}, av[4] = {0.f, 0.f, 0.f, 0.f};
         for (int i0 = 0; i0 < d; i0 += 1024) {
             const int span = d - i0 < 1024 ? d - i0 : 1024;
             __syncthreads();
@@ -173,33 +170,43 @@ __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *co
                 }
             }
             __syncthreads();
-            if (!live) continue;
-            for (int i = lane * NV; i < span; i += 32 * NV) {
-                float w[NV];
-                WVec<TS>::load(wrow + i0 + i, w);
+            // every warp takes MODW_OUT / 8 outputs; a row wider than 1024 is summed in parts (kept in uv itself)
+            for (int oi = 0; oi < MODW_OUT / 8; ++oi) {
+                const int o = o_cta + warp * (MODW_OUT / 8) + oi;
+                if (o >= 3 * d + dm) break;
+                const int oo = mlp ? o - 3 * d : o;
+                const TS *wrow = W + (size_t)oo * d + i0;
+                float au[4] = {0.f, 0.f, 0.f, 0.f}, av[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int i = lane * NV; i < span; i += 32 * NV) {
+                    float w[NV];
+                    WVec<TS>::load(wrow + i, w);
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (c0 + r < nc) {
+                    for (int r = 0; r < 4; ++r) {
+                        if (c0 + r < nc) {
 #pragma unroll
-                        for (int e = 0; e < NV; e += 4) {
-                            const float4 sc = *reinterpret_cast<const float4 *>(&s_sc[r][i + e]);
-                            const float4 sh = *reinterpret_cast<const float4 *>(&s_sh[r][i + e]);
-                            au[r] = fmaf(w[e], sc.x, au[r]), av[r] = fmaf(w[e], sh.x, av[r]);
-                            au[r] = fmaf(w[e + 1], sc.y, au[r]), av[r] = fmaf(w[e + 1], sh.y, av[r]);
-                            au[r] = fmaf(w[e + 2], sc.z, au[r]), av[r] = fmaf(w[e + 2], sh.z, av[r]);
-                            au[r] = fmaf(w[e + 3], sc.w, au[r]), av[r] = fmaf(w[e + 3], sh.w, av[r]);
+                            for (int e = 0; e < NV; e += 4) {
+                                const float4 sc = *reinterpret_cast<const float4 *>(&s_sc[r][i + e]);
+                                const float4 sh = *reinterpret_cast<const float4 *>(&s_sh[r][i + e]);
+                                au[r] = fmaf(w[e], sc.x, au[r]), av[r] = fmaf(w[e], sh.x, av[r]);
+                                au[r] = fmaf(w[e + 1], sc.y, au[r]), av[r] = fmaf(w[e + 1], sh.y, av[r]);
+                                au[r] = fmaf(w[e + 2], sc.z, au[r]), av[r] = fmaf(w[e + 2], sh.z, av[r]);
+                                au[r] = fmaf(w[e + 3], sc.w, au[r]), av[r] = fmaf(w[e + 3], sh.w, av[r]);
+                            }
                         }
                     }
                 }
-            }
-        }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            if (c0 + r >= nc) break;
-            const float su = warp_sum(au[r]), sv = warp_sum(av[r]);
-            if (lane == 0 && live)
-                uv[(size_t)sp->cd[c0 + r].slot * uv_row_stride + (size_t)layer * (3 * d + dm) + o] =
-                    make_float2(su, sv + bo);
+                for (int r = 0; r < 4; ++r) {
+                    if (c0 + r >= nc) break;
+                    float su = warp_sum(au[r]), sv = warp_sum(av[r]);
+                    float2 *dst = uv + (size_t)sp->cd[c0 + r].slot * uv_row_stride + (size_t)layer * (3 * d + dm) + o;
+                    if (lane == 0) {
+                        if (i0 > 0) su += dst->x, sv += dst->y;          // this thread wrote the earlier part itself
+                        if (i0 + span >= d) sv += to_f(B[oo]);
+                        *dst = make_float2(su, sv);
+                    }
+                }
+            }
         }
     }
     NFD_TRACE_END(TRK_GEMV);
