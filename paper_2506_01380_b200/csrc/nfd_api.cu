@@ -409,6 +409,147 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     }
 }
 
+// ---------------------------------------------------------------------------
+// Tile width and split of the four GEMMs of a block, found by timing at create.  For a pass of one frame
+// every (width, split) pair is timed and the best split is kept for good (the order in which the K range is
+// summed must not depend on the pass); for passes of more frames only the width is timed.  Results are kept
+// per process (nfd_fast.cuh), so a second context of the same shape does not time anything and sums in the
+// same order.  The timed launches run the real epilogues on scratch frames 0..nf-1 of stream 0 with whatever
+// the modulation tables hold; the caller clears the cache afterwards.
+// ---------------------------------------------------------------------------
+static int tune_gemms(nfd_ctx *c) {
+    const Dims &D = c->D;
+    const int d = D.d, T = D.T;
+    FastState &fs = c->fs;
+    if (!c->bf16_mode || !c->fast || !fs.ready || getenv("NFD_NO_TUNE") || getenv("NFD_GEMM_PLAN")) return NFD_OK;
+    const bool fold = c->fold_active();
+    const size_t mod_row = (size_t)D.L * 6 * d, uv_row = (size_t)D.L * (3 * d + D.n1);
+    struct Kind { int tc, N, K; };
+    const Kind kinds[4] = {{TC_QKV, 3 * d, d}, {TC_RES, d, d}, {TC_GELU, D.n1, d}, {TC_RES, d, D.dm}};
+    cudaEvent_t e0, e1;
+    CK(cudaEventCreate(&e0));
+    CK(cudaEventCreate(&e1));
+    const StepParams *sp = c->d_sp;
+    auto launch = [&](int ki, int M) -> bool {        // one launch of GEMM `ki` of layer 0 with the forced plan
+        const L2Prefetch pf{nullptr, 0};
+        const float *modl = c->mod;
+        LnFold ln{nullptr, uv_row, c->ln_stats, d / 32, D.norm, D.eps, sp, T};
+        if (ki == 0) {
+            if (fold) ln.uv = c->uvtab;
+            EpiQKV<bf16> e{sp, (const bf16 *)c->b_qkv[0], (bf16 *)c->qbuf, (bf16 *)c->kc, (bf16 *)c->vc, c->d_rope, D, 0,
+                           c->rope_cs, M, ln};
+            return fast_gemm<bf16>(true, fs, c->st, (const bf16 *)c->hbuf, (const bf16 *)c->w_qkv[0], M, 3 * d, d, e, TC_QKV, pf);
+        }
+        if (ki == 1) {
+            EpiGateRes<bf16> e{sp, (const bf16 *)c->b_o[0], c->z, modl + 2 * d, mod_row, D,
+                               fold ? (bf16 *)c->hbuf : (bf16 *)nullptr, modl + 4 * d, fold ? c->ln_stats : (float2 *)nullptr};
+            return fast_gemm<bf16>(true, fs, c->st, (const bf16 *)c->abuf, (const bf16 *)c->w_o[0], M, d, d, e, TC_RES, pf);
+        }
+        if (ki == 2) {
+            if (fold) ln.uv = c->uvtab + 3 * d;
+            EpiGelu<bf16> e{(const bf16 *)c->b_fc1[0], (bf16 *)c->mbuf, D.n1, D.act, ln};
+            return fast_gemm<bf16>(true, fs, c->st, (const bf16 *)c->hbuf, (const bf16 *)c->w_fc1[0], M, D.n1, d, e, TC_GELU, pf);
+        }
+        EpiGateRes<bf16> e{sp, (const bf16 *)c->b_fc2[0], c->z, modl + 5 * d, mod_row, D,
+                           fold ? (bf16 *)c->hbuf : (bf16 *)nullptr, modl + 7 * d, fold ? c->ln_stats : (float2 *)nullptr};
+        return fast_gemm<bf16>(true, fs, c->st, (const bf16 *)c->mbuf, (const bf16 *)c->w_fc2[0], M, d, D.dm, e, TC_RES, pf);
+    };
+    auto time_of = [&](int ki, int M, int BN, int S, float *us) -> bool {
+        fs.force_BN = BN, fs.force_S = S;
+        bool ok = true;
+        for (int i = 0; i < 3 && ok; ++i) ok = launch(ki, M);
+        float best = 1e30f;
+        for (int rep = 0; rep < 3 && ok; ++rep) {
+            cudaEventRecord(e0, c->st);
+            for (int i = 0; i < 8 && ok; ++i) ok = launch(ki, M);
+            cudaEventRecord(e1, c->st);
+            if (cudaEventSynchronize(e1) != cudaSuccess) ok = false;
+            float ms = 0.f;
+            if (ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && ms < best) best = ms;
+        }
+        fs.force_BN = fs.force_S = 0;
+        if (!ok) cudaGetLastError();
+        *us = best * 1000.f / 8.f;
+        return ok;
+    };
+    const int nfs[] = {1, 2, 3, 4, 5, 6, 8, 12, 16, 24, 32};
+    const int widths[] = {32, 64, 96, 128, 192, 256};
+    bool touched = false;
+    // the largest pass this context can build: per stream a speculation plus the deferred frames of the last one
+    const int nf_max = D.n_streams * 2 * c->cfg.max_spec;
+    for (int nf : nfs) {
+        if (nf > NFD_MAX_PASS_FRAMES || nf > nf_max) break;
+        const int M = nf * T;
+        bool need = false;
+        for (const Kind &k : kinds)
+            if (!g_tuned_BN.count(std::make_tuple(k.tc + (k.K > 2048 ? 10 : 0), k.N, k.K, fs.n_sm, M))) need = true;
+        if (!need) continue;
+        // a pass descriptor for nf scratch frames of stream 0
+        StepParams &p = c->h_sp;
+        memset(&p, 0, sizeof(p));
+        p.nf = nf;
+        for (int j = 0; j < nf; ++j) {
+            p.fr[j].stream = 0, p.fr[j].frame = j, p.fr[j].win_first = 0, p.fr[j].cond_row = 0, p.fr[j].first_new = 0;
+            p.fr[j].src = 0, p.fr[j].src_index = j, p.fr[j].out_index = -1;
+        }
+        k_set_params<<<1, 256, 0, c->st>>>(p, c->d_sp);
+        CK(cudaGetLastError());
+        touched = true;
+        for (int ki = 0; ki < 4; ++ki) {
+            const Kind &k = kinds[ki];
+            const int kk = k.tc + (k.K > 2048 ? 10 : 0);
+            const auto skey = std::make_tuple(kk, k.N, k.K, fs.n_sm);
+            const auto bkey = std::make_tuple(kk, k.N, k.K, fs.n_sm, M);
+            if (g_tuned_BN.count(bkey)) continue;
+            const bool s_open = !g_tuned_S.count(skey);
+            if (s_open && nf != 1) continue;                 // the split is decided by the one-frame pass
+            const int nkb = (k.K + 63) / 64;
+            // the cost model's plan is the incumbent: another one must beat it by 3 % (timing noise must not
+            // flip plans between processes without need)
+            const GemmPlan model = plan_gemm(fs, M, k.N, k.K, k.tc);
+            float t_best = 1e30f;
+            GemmPlan best = model;
+            if (!time_of(ki, M, model.BN, model.S, &t_best)) t_best = 1e30f;
+            if (getenv("NFD_TUNE_LOG") && nf <= 2)
+                fprintf(stderr, "libnfd:   kind %d M %d model BN %d S %d: %.2f us\n", kk, M, model.BN, model.S, t_best);
+            t_best *= 0.97f;
+            for (int S = 1; S <= 4; S *= 2) {
+                if (!s_open && S != g_tuned_S[skey]) continue;
+                if (S > 1 && nkb / S < 2) continue;
+                for (int BN : widths) {
+                    if (BN > 32 && BN > k.N) continue;
+                    if (nf == 1 && BN > 128) continue;
+                    if (BN == model.BN && S == model.S) continue;
+                    const long long ctas = (long long)((M + 127) / 128) * ((k.N + BN - 1) / BN) * S;
+                    if (ctas > 3LL * fs.n_sm) continue;          // hopeless: several waves
+                    float t;
+                    const bool ok_t = time_of(ki, M, BN, S, &t);
+                    if (getenv("NFD_TUNE_LOG") && nf <= 2)
+                        fprintf(stderr, "libnfd:   kind %d M %d BN %d S %d: %.2f us%s\n", kk, M, BN, S, t, ok_t ? "" : " (failed)");
+                    if (ok_t && t < t_best) t_best = t, best = GemmPlan{BN, S};
+                }
+            }
+            if (s_open) g_tuned_S[skey] = best.S;
+            g_tuned_BN[bkey] = best.BN;
+            if (getenv("NFD_TUNE_LOG"))
+                fprintf(stderr, "libnfd: tuned kind %d N %d K %d M %d -> BN %d S %d (model BN %d S %d)\n", kk, k.N, k.K, M,
+                        best.BN, best.S, model.BN, model.S);
+        }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (touched) {
+        // the timed epilogues wrote into scratch pages of stream 0 and into the activation buffers
+        const size_t cache_bytes = (size_t)D.n_streams * D.L * D.R * D.page_elems * c->esz;
+        CK(cudaMemsetAsync(c->kc, 0, cache_bytes, c->st));
+        CK(cudaMemsetAsync(c->vc, 0, cache_bytes, c->st));
+        CK(cudaMemsetAsync(c->d_status, 0, 4, c->st));
+        CK(cudaStreamSynchronize(c->st));
+        memset(&c->h_sp, 0, sizeof(c->h_sp));
+    }
+    return NFD_OK;
+}
+
 static void enqueue_body_any(nfd_ctx *c, int nf, int kind) {
     if (c->bf16_mode)
         enqueue_body<bf16>(c, nf, kind);
@@ -708,6 +849,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
         }
     }
     if (rc == NFD_OK) rc = fast_create(c->fs, D, c->bf16_mode, c->st, c->d_status);
+    if (rc == NFD_OK) rc = tune_gemms(c);
     if (rc != NFD_OK) {
         nfd_destroy(c);
         return rc;
