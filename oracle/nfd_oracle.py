@@ -95,6 +95,49 @@ def renoise(x0, z, tp_next: float, sigma_d: float):
     return math.cos(tp_next) * np.asarray(x0, F64) + math.sin(tp_next) * sigma_d * np.asarray(z, F64)
 
 
+def dpmpp_grid(n_evals: int):
+    """Time grid of the multistep ODE sampler below: t_0 = 1 (pure noise) down to t_M = 0 in M = n_evals equal
+    steps of Flow-Matching time; the model is evaluated at t_0 .. t_{M-1}.  (Section 3.2 "Sampling" names the
+    solver and, in the experiments, 18 function evaluations; it gives no grid, so equal steps are a reading.)"""
+    return [1.0 - i / n_evals for i in range(n_evals + 1)]
+
+
+def dpmpp_coeffs(t_prev2, t_prev: float, t: float, last: bool):
+    """Coefficients (a, b, c) of one step t_prev -> t of DPM-Solver++(2M) (Lu et al. 2022, the multistep
+    second-order solver for data-prediction models), written for the Flow-Matching path alpha_t = 1 - t,
+    sigma_t = t, lambda_t = ln(alpha_t / sigma_t):
+        x_t = (sigma_t / sigma_prev) x_prev - alpha_t (exp(-h) - 1) D,   h = lambda_t - lambda_prev,
+        D   = (1 + 1/(2r)) x0(t_prev) - 1/(2r) x0(t_prev2),              r = h_prev / h,
+    returned as x_t = a x_prev + b ((1 + c) x0(t_prev) - c x0(t_prev2)).  Where a lambda is infinite (t = 1 at the
+    start, t = 0 at the end) the limits are taken: exp(-h) -> 0, and the step is first order (c = 0) when there is
+    no finite previous step, which is the first two steps; the last step is first order as well (the customary
+    "lower order final" rule; with t = 0 it returns the last data prediction itself)."""
+    a = t / t_prev
+    # -alpha_t (exp(-h) - 1) with exp(-h) = (alpha_prev / sigma_prev) (sigma_t / alpha_t)
+    b = (1.0 - t) - (1.0 - t_prev) * t / t_prev
+    c = 0.0
+    if t_prev2 is not None and not last and t_prev2 < 1.0 and t > 0.0:
+        lam = lambda u: math.log((1.0 - u) / u)
+        h, h_prev = lam(t) - lam(t_prev), lam(t_prev) - lam(t_prev2)
+        c = h / (2.0 * h_prev)              # 1 / (2 r)
+    return a, b, c
+
+
+def dpmpp_2m(x0_fn, x_T, n_evals: int):
+    """DPM-Solver++(2M) over dpmpp_grid from x_T (at t = 1) to t = 0 for a data-prediction function
+    x0_fn(x, t).  Returns the sample at t = 0."""
+    ts = dpmpp_grid(n_evals)
+    x = np.asarray(x_T, F64)
+    x0_prev = None
+    for i in range(1, n_evals + 1):
+        x0_cur = x0_fn(x, ts[i - 1])
+        a, b, c = dpmpp_coeffs(ts[i - 2] if i >= 2 else None, ts[i - 1], ts[i], last=(i == n_evals))
+        D = (1.0 + c) * x0_cur - (c * x0_prev if c != 0.0 else 0.0)
+        x = a * x + b * D
+        x0_prev = x0_cur
+    return x
+
+
 def accepted_count(true_actions, i: int, k: int) -> int:
     """Section 4.2 / appendix listing: frames i..i+k-1 were generated under
     action true_actions[i] repeated.  The leading frames whose true action
@@ -402,6 +445,18 @@ class NFDOracle:
             x0 = f_theta(x, F_theta(x_in, v, t), tp, self.sigma_d)
             if s + 1 < S:
                 x = renoise(x0, noise[s + 1], sched[s + 1], self.sigma_d)
+        self._commit(x0, [action] * k, ctx_noise, tentative=True)
+        return x0
+
+    def sample_dpmpp(self, k: int, action: int, noise, n_evals: int = 18, ctx_noise=None):
+        """The undistilled sampler of Section 3.2 "Sampling": the Flow-Matching model integrated from pure noise
+        with DPM-Solver++ (n_evals function evaluations, 18 in the paper's experiments) for k frames decoded
+        together under `action`; the clean frames are appended to the cache as tentative.  noise [k,C,H,W] in
+        unit variance; latents are in units of sigma_d, so the model sees x/sigma_d.  Data prediction from the
+        velocity: x0 = x_t - t v (Section 3.2).  Returns x0 [k,C,H,W]."""
+        def x0_fn(x, t):
+            return x - t * self.denoise_step(x, t, action)
+        x0 = self.sigma_d * dpmpp_2m(x0_fn, np.asarray(noise, F64), n_evals)
         self._commit(x0, [action] * k, ctx_noise, tentative=True)
         return x0
 
