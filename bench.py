@@ -275,6 +275,8 @@ def main():
     ap.add_argument("--workload", default="nfd310m", choices=sorted(WORKLOADS),
                     help="nfd310m is the configuration the metric is quoted on; the others are the paper's own "
                          "size-table shapes with a gated MLP (second workload, same step definition)")
+    ap.add_argument("--dpmpp", action="store_true",
+                    help="add the undistilled sampler leg (DPM-Solver++, 18 function evaluations per frame)")
     ap.add_argument("--batch8", action="store_true",
                     help="add the 8-stream, 32-frame-context leg (aggregate and per-stream frames/s)")
     ap.add_argument("--spec-sweep", action="store_true",
@@ -426,6 +428,27 @@ def main():
         line["spec_k4"] = {"accepted_frames_per_s": round(acc / (ms4 * 1e-3), 3), "acceptance_rate": round(acc / spec, 4),
                            "accepted_per_pass": round(acc / passes, 4), "ms_per_speculate": round(ms4 / passes, 4),
                            "p_repeat": 0.8, "frames": acc}
+
+        # ---------------- the undistilled sampler: 18 evaluations of the model per frame + commit ----------------
+        if args.dpmpp:
+            n_d = 16
+            fill_prompt()
+            zn, zc = randn(1, *fs), randn(1, *fs)
+            with torch.cuda.stream(nfd.stream):
+                for i in range(2):
+                    nfd.sample_dpmpp(1, actions[i], zn, n_evals=18, ctx_noise=zc, out=x0)
+                    nfd.rollback(1)
+                torch.cuda.synchronize(device)
+                e0.record(nfd.stream)
+                for i in range(n_d):
+                    nfd.sample_dpmpp(1, actions[i], zn, n_evals=18, ctx_noise=zc, out=x0)
+                    nfd.rollback(1)
+                e1.record(nfd.stream)
+                torch.cuda.synchronize(device)
+            ms_d = e0.elapsed_time(e1)
+            line["dpmpp18"] = {"frames_per_s": round(n_d / (ms_d * 1e-3), 3), "ms_per_frame": round(ms_d / n_d, 3),
+                               "n_evals": 18, "forward_passes_per_frame": 19, "steps": n_d,
+                               "paper_context_fps_a100": {"nfd310m": 6.15}.get(args.workload)}
 
         # ---------------- 8 independent streams, 32-frame context, one batched call per frame ----------------
         if args.batch8:

@@ -239,6 +239,17 @@ int nfd_profile_end(nfd_ctx *ctx, int n_classes, long long *n_launches, float *t
 int nfd_profile_class_count(void);
 const char *nfd_profile_class_name(int id);
 
+/* The undistilled sampler of Section 3.2 "Sampling": the Flow-Matching model integrated from pure noise with
+ * DPM-Solver++ (the multistep second-order solver for data-prediction models; data prediction x0 = x_t - t v)
+ * in n_evals function evaluations (18 in the paper's experiments) for k frames decoded together under
+ * `action`.  The paper gives neither grid nor order: equal steps of FM time from 1 to 0, second order except
+ * for the first two steps (no finite previous step: lambda is infinite at t = 1) and the last one.
+ * noise dev [k,C,H,W] (unit variance), ctx_noise dev [k,C,H,W] or NULL, x0_out dev [k,C,H,W].  Like
+ * nfd_speculate it leaves the k frames in the cache as tentative (committed at once, not deferred); pending
+ * frames of the stream are written first.  Errors as nfd_speculate; n_evals outside 1..1000: NFD_E_RANGE. */
+int nfd_sample_dpmpp(nfd_ctx *ctx, int stream, int k, int action, int n_evals, const float *noise,
+                     const float *ctx_noise, float *x0_out);
+
 /* Fills the modulation cache for every (time, action) pair that nfd_speculate
  * and the commits can ask for: the n_steps sampler times (Section 4.1
  * "Sampling") and the context time (Section 4.3), each with every action.  The

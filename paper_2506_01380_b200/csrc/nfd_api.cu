@@ -61,6 +61,7 @@ struct nfd_ctx {
     void *hbuf = nullptr, *qbuf = nullptr, *abuf = nullptr, *mbuf = nullptr;
     float *emb = nullptr, *h1 = nullptr, *sc = nullptr, *mod = nullptr, *fmod = nullptr;
     float *xp = nullptr, *vbuf = nullptr;       // sampler state, velocity
+    float *x0_prev = nullptr;                   // previous data prediction of the multistep ODE sampler
     float2 *rope_cs = nullptr;                  // per-pass RoPE table [Nq_max][dh/2]
     StepParams *d_sp = nullptr;
     StepParams h_sp;
@@ -811,6 +812,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     A((void **)&c->pend_cz, (size_t)cfg->n_streams * cfg->max_spec * c->frame_elems() * 4);
     A((void **)&c->xp, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->vbuf, (size_t)NF * c->frame_elems() * 4);
+    A((void **)&c->x0_prev, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->d_sp, sizeof(StepParams));
     A((void **)&c->d_hash, 8);
     A((void **)&c->d_status, 4);
@@ -1115,6 +1117,48 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
         c->n_tentative[st] += k;
     }
     return NFD_OK;
+}
+
+// The undistilled sampler (Section 3.2 "Sampling"): DPM-Solver++(2M) over n_evals equal steps of FM time from
+// t = 1 (pure noise) to t = 0; first order where no finite previous step exists (the first two steps) and at
+// the last step.  Coefficients as in the published algorithm, with alpha_t = 1 - t, sigma_t = t.
+int nfd_sample_dpmpp(nfd_ctx *c, int stream, int k, int action, int n_evals, const float *noise,
+                     const float *ctx_noise, float *x0_out) {
+    if (!c) return NFD_E_NULLPTR;
+    RET(check_io(noise, x0_out));
+    if (!aligned16(ctx_noise)) return NFD_E_ALIGN;
+    if (stream < 0 || stream >= c->cfg.n_streams) return NFD_E_RANGE;
+    if (k < 1 || k > c->cfg.max_spec || n_evals < 1 || n_evals > 1000) return NFD_E_RANGE;
+    if (action < 0 || action >= c->cfg.n_actions) return NFD_E_RANGE;
+    if (c->n_tentative[stream] != 0) return NFD_E_STATE;
+    RET(flush_pending(c, stream));
+    const size_t ne = (size_t)k * c->frame_elems();
+    const int eg = (int)((ne + 255) / 256);
+    c->cls = CLS_SAMPLER;
+    PLAUNCH(c, k_axpby, eg, 256, 0, c->xp, 1.0f, noise, 0.f, (const float *)nullptr, ne);
+    const int M = n_evals;
+    auto tgrid = [M](int i) { return 1.0 - (double)i / (double)M; };
+    auto lam = [](double u) { return log((1.0 - u) / u); };
+    for (int i = 1; i <= M; ++i) {
+        const double tp = tgrid(i - 1), tn = tgrid(i);
+        const float tf = (float)tp;
+        RET(build_pass(c, 1, &stream, k, 0, &tf, &action, false, 0, c->xp, 1.0f, nullptr, 0.f, c->vbuf));
+        RET(run_pass(c));
+        const double a = tn / tp;
+        const double b = (1.0 - tn) - (1.0 - tp) * tn / tp;
+        double cc = 0.0;
+        if (i >= 3 && i < M) {                // a finite previous step exists and this is not the last step
+            const double tpp = tgrid(i - 2);
+            cc = (lam(tn) - lam(tp)) / (2.0 * (lam(tp) - lam(tpp)));
+        }
+        c->cls = CLS_SAMPLER;
+        PLAUNCH(c, k_dpmpp_update, eg, 256, 0, c->xp, (const float *)c->vbuf, c->x0_prev, tf, (float)a, (float)b,
+                (float)cc, i == M ? x0_out : (float *)nullptr, c->cfg.sigma_d, ne);
+    }
+    CK(cudaGetLastError());
+    CK(c->launch_err);
+    std::vector<int> fa(k, action);
+    return commit_pass(c, 1, &stream, k, fa.data(), x0_out, ctx_noise, true);
 }
 
 int nfd_speculate(nfd_ctx *c, int stream, int k, int action, const float *noise, const float *ctx_noise,

@@ -879,6 +879,25 @@ __global__ void k_sampler_post(float *xp, const float *v, const float *z, float 
     if (z) xp[i] = fmaf(s, z[i], c * e);
 }
 
+// One step of DPM-Solver++(2M) on the Flow-Matching path (Section 3.2 "Sampling" names the solver; the update
+// is the published multistep form with data prediction x0 = x - t v):
+//     x <- a x + b ((1 + c) x0 - c x0_prev),   x0_prev <- x0;   out = scale * x  when out is given (last step).
+__global__ void k_dpmpp_update(float *x, const float *v, float *x0_prev, float t, float a, float b, float c,
+                               float *out, float scale, size_t n) {
+    pdl_wait();
+    pdl_launch();
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float xi = x[i];
+    const float x0 = fmaf(-t, v[i], xi);
+    float D = x0;
+    if (c != 0.f) D = fmaf(c, x0 - x0_prev[i], x0);
+    const float xn = fmaf(b, D, a * xi);
+    x[i] = xn;
+    x0_prev[i] = x0;
+    if (out) out[i] = scale * xn;
+}
+
 // ---------------------------------------------------------------------------
 // Cache read-out, fill and digest.
 // ---------------------------------------------------------------------------

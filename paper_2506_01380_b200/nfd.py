@@ -44,7 +44,8 @@ EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_de
            "nfd_rollback", "nfd_kv_state", "nfd_kv_hash", "nfd_kv_read", "nfd_attention", "nfd_status",
            "nfd_launch_count", "nfd_set_option", "nfd_warm_modulation", "nfd_strerror", "nfd_profile_begin",
            "nfd_profile_end",
-           "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc", "nfd_cond_cache_stats"]
+           "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc", "nfd_cond_cache_stats",
+           "nfd_sample_dpmpp"]
 
 
 class NfdError(RuntimeError):
@@ -74,6 +75,7 @@ def load():
     lib.nfd_commit_frame.argtypes = [vp, C.c_int, vp, C.c_int, ip, vp]
     lib.nfd_speculate.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     lib.nfd_speculate_batched.argtypes = [vp, C.c_int, ip, C.c_int, ip, vp, vp, vp]
+    lib.nfd_sample_dpmpp.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     lib.nfd_rollback.argtypes = [vp, C.c_int, C.c_int]
     lib.nfd_kv_state.argtypes = [vp, C.c_int, ip, ip, ip]
     lib.nfd_kv_hash.argtypes = [vp, C.c_int, C.POINTER(C.c_ulonglong)]
@@ -252,6 +254,16 @@ class NFD:
         _check(self.lib.nfd_speculate(self._h, stream, k, int(action), self._f32(noise, (S, k) + self.frame_shape),
                                       self._f32(ctx_noise, x0.shape) if ctx_noise is not None else None,
                                       self._f32(x0)), "nfd_speculate")
+        self._exit()
+        return x0
+
+    def sample_dpmpp(self, k: int, action: int, noise, n_evals: int = 18, ctx_noise=None, stream: int = 0, out=None):
+        x0 = torch.empty((k,) + self.frame_shape, device=self.device, dtype=torch.float32) if out is None else out
+        self._enter()
+        _check(self.lib.nfd_sample_dpmpp(self._h, stream, k, int(action), int(n_evals),
+                                         self._f32(noise, (k,) + self.frame_shape),
+                                         self._f32(ctx_noise, x0.shape) if ctx_noise is not None else None,
+                                         self._f32(x0)), "nfd_sample_dpmpp")
         self._exit()
         return x0
 

@@ -331,6 +331,37 @@ def test_modulation_cache_hits_evictions_and_values():
     assert g.status() == 0
 
 
+@pytest.mark.parametrize("name,kind,n_evals", [("tiny", "stress", 18), ("tiny", "paper", 5), ("tiny_bf16", "paper", 18),
+                                               ("tiny_gated_bf16", "stress", 6)])
+def test_dpmpp_sampler_matches_oracle(name, kind, n_evals):
+    """The undistilled sampler (DPM-Solver++ over n_evals evaluations of the Flow-Matching model): generated
+    frames, counters and the tentative K/V pages against the oracle, then rollback."""
+    cfg = I.make_cfg(name)
+    g, orc = make_pair(cfg, 21, kind)
+    prompt(cfg, g, orc, 3, seed=300, group=3)
+    k = 2
+    noise = I.make_latents(cfg, k, 310)
+    cz = I.make_latents(cfg, k, 311)
+    if cfg["dtype"] == I.DTYPE_BF16:
+        noise, cz = I.round_bf16(noise), I.round_bf16(cz)
+    y = g.sample_dpmpp(k, 5, dev(noise), n_evals=n_evals, ctx_noise=dev(cz))
+    ref = orc.sample_dpmpp(k, 5, noise.astype(np.float64), n_evals=n_evals, ctx_noise=cz.astype(np.float64))
+    check(y, ref, cfg["dtype"], "x0")
+    assert g.kv_state() == (orc.n_committed, orc.n_tentative, orc.window_first())
+    assert g.kv_state()[:2] == (3, k)
+    for l in range(cfg["n_layers"]):
+        for f in (3, 4):
+            K, V = g.kv_read(l, f)
+            check(K, orc.kv_frame(l, f)[0], cfg["dtype"], f"K l{l} f{f}", scale_by_magnitude=True)
+            check(V, orc.kv_frame(l, f)[1], cfg["dtype"], f"V l{l} f{f}", scale_by_magnitude=True)
+    g.rollback(1), orc.rollback(1)
+    assert g.kv_state() == (orc.n_committed, orc.n_tentative, orc.window_first())
+    assert g.kv_state()[:2] == (4, 0)
+    with pytest.raises(Exception):
+        g.sample_dpmpp(k, 5, dev(noise), n_evals=0)
+    assert g.status() == 0
+
+
 @pytest.mark.parametrize("name", ["tiny_bf16", "tiny"])
 def test_warm_modulation_fills_every_schedule_pair(name):
     """nfd_warm_modulation computes the modulation of all (sampler or context time, action) pairs up front:
