@@ -36,6 +36,10 @@ struct AttnPlan {
     int MAXSPLIT = 0;    // splits of the longest window
 };
 
+#ifndef ATTN_POLY_PAIR
+#define ATTN_POLY_PAIR (-1)     // which of the 4 column pairs of an 8-column group uses ex2_poly (-1: none)
+#endif
+
 template <int KB> struct AttnCfg {
     static constexpr int NST = 4;                          // K/V ring stages
     static constexpr int Q_BYTES = 128 * 128;
@@ -58,6 +62,41 @@ __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// 2^y on the FMA and integer pipes, for a share of the softmax's exponentials: the special-function unit
+// (16 ex2 per clock and SM) is what bounds the softmax at head dimension 64.  Round-to-nearest split
+// y = n + f by the magic-number addition, a cubic for 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below
+// the bf16 rounding of P), n added to the exponent field.  y <= 127; results below 2^-125 are clamped there.
+__device__ __forceinline__ float ex2_poly(float y) {
+    y = fmaxf(y, -125.0f);
+    const float t = y + 12582912.0f;               // 1.5 * 2^23: round(y) lands in the low mantissa bits
+    const float f = y - (t - 12582912.0f);
+    float p = fmaf(0.05517220f, f, 0.24261118f);
+    p = fmaf(p, f, 0.69326091f);
+    p = fmaf(p, f, 0.99992806f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// Two fp32 lanes per instruction (sm_100 f32x2 forms): d = a * b + c and d = a + b on register pairs.
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    unsigned long long ra, rb, rc, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
 }
 
 __device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
@@ -251,7 +290,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             }
             // pass 2 over S, 16 columns at a time with the next load in flight:
             // P = exp2(S c - m) as bf16 into shared memory (128-byte-swizzled K-major layout)
-            float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+            float2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
             uint32_t sa[16], sb[16];
             tmem_ld16(tS, sa);
 #pragma unroll
@@ -264,9 +303,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                     uint32_t pk[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(cur[8 * u2 + 2 * u]), c, -m_run));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(cur[8 * u2 + 2 * u + 1]), c, -m_run));
-                        ls4[u] += p0 + p1;
+                        // one pair in four goes to the FMA pipes (ex2_poly)
+                        const float2 y = ffma2(make_float2(__uint_as_float(cur[8 * u2 + 2 * u]),
+                                                           __uint_as_float(cur[8 * u2 + 2 * u + 1])),
+                                               make_float2(c, c), make_float2(-m_run, -m_run));
+                        const float p0 = (u == ATTN_POLY_PAIR) ? ex2_poly(y.x) : ex2_approx(y.x);
+                        const float p1 = (u == ATTN_POLY_PAIR) ? ex2_poly(y.y) : ex2_approx(y.y);
+                        ls2[u] = fadd2(ls2[u], make_float2(p0, p1));
                         const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
                         pk[u] = *reinterpret_cast<const uint32_t *>(&hp);
                     }
@@ -275,7 +318,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                     *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
-            l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+            l_run += ((ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y)) + ((ls2[2].x + ls2[2].y) + (ls2[3].x + ls2[3].y));
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(p_full + 8 * g);
