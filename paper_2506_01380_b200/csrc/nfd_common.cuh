@@ -157,6 +157,37 @@ __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x));
 __device__ __forceinline__ float silu_fast_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
 
+// Two fp32 lanes per instruction (sm_100 f32x2 forms): d = a * b + c and d = a + b on register pairs.
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    unsigned long long ra, rb, rc, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+
 // GELU (erf form) for values that are rounded to bf16 afterwards: erf by the
 // rational approximation 7.1.26 of Abramowitz & Stegun (absolute error below
 // 1.5e-7, three orders of magnitude under the bf16 rounding step).
@@ -170,6 +201,23 @@ __device__ __forceinline__ float gelu_erf_bf16_f(float x) {
     p = fmaf(p, t, 0.254829592f);
     const float e = fmaf(-p * t, __expf(-z * z), 1.0f);      // erf(|x|/sqrt 2)
     return 0.5f * fmaf(ax, e, x);                            // x/2 (1 + sign(x) e)
+}
+// the same for two values at once, on the two-lane fp32 instructions
+__device__ __forceinline__ float2 gelu_erf_bf16_f2(float2 x) {
+    const float2 ax = make_float2(fabsf(x.x), fabsf(x.y));
+    const float2 z = fmul2(ax, make_float2(0.70710678118654752440f, 0.70710678118654752440f));
+    const float2 den = ffma2(make_float2(0.3275911f, 0.3275911f), z, make_float2(1.0f, 1.0f));
+    const float2 t = make_float2(__fdividef(1.0f, den.x), __fdividef(1.0f, den.y));
+    float2 p = ffma2(make_float2(1.061405429f, 1.061405429f), t, make_float2(-1.453152027f, -1.453152027f));
+    p = ffma2(p, t, make_float2(1.421413741f, 1.421413741f));
+    p = ffma2(p, t, make_float2(-0.284496736f, -0.284496736f));
+    p = ffma2(p, t, make_float2(0.254829592f, 0.254829592f));
+    const float2 nzz = fmul2(fmul2(z, z), make_float2(-1.0f, -1.0f));
+    const float2 ex = make_float2(__expf(nzz.x), __expf(nzz.y));
+    const float2 npt = fmul2(fmul2(p, t), make_float2(-1.0f, -1.0f));
+    const float2 e = ffma2(npt, ex, make_float2(1.0f, 1.0f));
+    const float2 r = ffma2(ax, e, x);
+    return fmul2(r, make_float2(0.5f, 0.5f));
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

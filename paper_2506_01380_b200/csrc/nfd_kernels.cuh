@@ -695,7 +695,10 @@ template <typename TS> struct EpiGelu {
             bias_add(a, s.bias);
         if (act == 0) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a[i] = gelu_erf_bf16_f(a[i]);
+            for (int i = 0; i < 8; i += 2) {
+                const float2 g = gelu_erf_bf16_f2(make_float2(a[i], a[i + 1]));
+                a[i] = g.x, a[i + 1] = g.y;
+            }
             *reinterpret_cast<uint4 *>(out + (size_t)m * N + n) = pack_bf16x8(a);
         } else {
             uint2 o;
