@@ -107,6 +107,28 @@ def test_denoise_step_after_prompt(name, kind, opts):
     assert g.launch_count() > 0
 
 
+@pytest.mark.parametrize("name,opts", [("tiny", {}), ("tiny_bf16", {}), ("tiny_bf16", {"fuse_ln": 0}),
+                                       ("tiny_bf16", {"fast": 0}), ("tiny_gated_bf16", {})])
+def test_rmsnorm_variant(name, opts):
+    """cfg.norm = 1: RMSNorm instead of LayerNorm in every adaLN (no mean removal), on every path: fp32
+    validation kernels, bf16 with the norm folded into the GEMMs, bf16 with stand-alone norm kernels, bf16
+    plain kernels."""
+    cfg = I.make_cfg(name, norm=1)
+    g, orc = make_pair(cfg, 4, "stress", **opts)
+    prompt(cfg, g, orc, 3, seed=500, group=2)
+    x_t = I.make_latents(cfg, 2, 510)
+    if cfg["dtype"] == I.DTYPE_BF16:
+        x_t = I.round_bf16(x_t)
+    v = g.denoise_step(dev(x_t), 0.4375, 2)
+    check(v, orc.denoise_step(x_t.astype(np.float64), 0.4375, 2), cfg["dtype"], "velocity")
+    for l in range(cfg["n_layers"]):
+        for f in (2, 3, 4):
+            K, V = g.kv_read(l, f)
+            check(K, orc.kv_frame(l, f)[0], cfg["dtype"], f"K l{l} f{f}")
+            check(V, orc.kv_frame(l, f)[1], cfg["dtype"], f"V l{l} f{f}")
+    assert g.status() == 0
+
+
 @pytest.mark.parametrize("name,kind", [("tiny", "stress"), ("tiny_bf16", "stress")])
 def test_joint_pass_equals_sequential(name, kind):
     cfg = I.make_cfg(name)
