@@ -129,6 +129,22 @@ def test_rmsnorm_variant(name, opts):
     assert g.status() == 0
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16"])
+def test_head_dim_128(name):
+    """Head dimension 128 (two heads of a 256-wide model; rotary split 32/48/48): the GEMMs take the
+    tensor-core path, attention the plain kernel."""
+    cfg = I.make_cfg(name, d_model=256, n_heads=2, head_dim=128, d_mlp=512, rope_t=32, rope_h=48, rope_w=48)
+    g, orc = make_pair(cfg, 6, "stress")
+    prompt(cfg, g, orc, 5, seed=600, group=3)                 # one more frame than the window holds
+    x_t = I.make_latents(cfg, 1, 610)
+    if cfg["dtype"] == I.DTYPE_BF16:
+        x_t = I.round_bf16(x_t)
+    v = g.denoise_step(dev(x_t), 0.6, 1)
+    check(v, orc.denoise_step(x_t.astype(np.float64), 0.6, 1), cfg["dtype"], "velocity")
+    assert g.kv_state() == (orc.n_committed, orc.n_tentative, orc.window_first())
+    assert g.status() == 0
+
+
 @pytest.mark.parametrize("name,kind", [("tiny", "stress"), ("tiny_bf16", "stress")])
 def test_joint_pass_equals_sequential(name, kind):
     cfg = I.make_cfg(name)
