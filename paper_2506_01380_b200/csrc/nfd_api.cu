@@ -851,6 +851,14 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
         }
     }
     if (rc == NFD_OK) rc = fast_create(c->fs, D, c->bf16_mode, c->st, c->d_status);
+    if (rc == NFD_OK && c->fs.ready) {
+        // how many CTAs of a GEMM fit at once, per cluster size (any instantiation: one CTA fills an SM)
+        auto kern = k_gemm_tc<96, EpiGateRes<bf16>, 0>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<96>::SMEM) == cudaSuccess)
+            query_gemm_slots(c->fs, kern, GemmCfg<96>::SMEM, GemmCfg<96>::THREADS);
+        else
+            cudaGetLastError();
+    }
     if (rc == NFD_OK) rc = tune_gemms(c);
     if (rc != NFD_OK) {
         nfd_destroy(c);

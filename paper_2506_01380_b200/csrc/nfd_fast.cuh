@@ -30,6 +30,7 @@ struct FastState {
     size_t cache_rows = 0;
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;   // (ptr, rows, cols, box_rows)
     int force_BN = 0, force_S = 0;     // set while candidates are being timed
+    int slots[5] = {0, 0, 0, 0, 0};    // CTAs of a GEMM that can be resident at once, by cluster size (1, 2, 4)
 };
 
 static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_t st, int *d_status) {
@@ -152,11 +153,27 @@ static std::map<std::tuple<int, int, int, int>, int> g_tuned_S;
 static std::map<std::tuple<int, int, int, int, int>, int> g_tuned_BN;
 
 // CTAs that can be resident at once: one per SM, less what clusters cannot use (a cluster lives inside one
-// GPC; measured here: 36 clusters of 4 did not fit at once, 33 did).
-static int gemm_slots(int n_sm, int S) {
-    if (S >= 4) return (n_sm / 4 - 4) * 4;
-    if (S == 2) return (n_sm / 2 - 2) * 2;
-    return n_sm;
+// GPC).  Asked of the runtime at create (on a 148-SM B200: 148 for clusters of 1 and 2, 132 for clusters of
+// 4); the fallback figures are those.
+static int gemm_slots(const FastState &fs, int S) {
+    if (S >= 1 && S <= 4 && fs.slots[S] > 0) return fs.slots[S];
+    if (S >= 4) return (fs.n_sm / 4 - 4) * 4;
+    return fs.n_sm;
+}
+template <typename Kern> static void query_gemm_slots(FastState &fs, Kern kern, int smem, int threads) {
+    for (int cs = 1; cs <= 4; cs *= 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(fs.n_sm / cs * cs), cfg.blockDim = dim3(threads), cfg.dynamicSmemBytes = (size_t)smem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = cs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+        cfg.attrs = at, cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0)
+            fs.slots[cs] = n * cs < fs.n_sm ? n * cs : fs.n_sm;
+        else
+            cudaGetLastError();
+    }
 }
 
 static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind) {
@@ -185,7 +202,7 @@ static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind)
     auto cost_of = [&](int m_rows, int BN, int S) {
         const int mt = (m_rows + 127) / 128, nt = (N + BN - 1) / BN;
         const long long ctas = (long long)mt * nt * S;
-        const int slots = gemm_slots(fs.n_sm, S);
+        const int slots = gemm_slots(fs, S);
         const double waves = (double)((ctas + slots - 1) / slots);
         const double share = 1.0;
         const double kb = (double)((nkb + S - 1) / S);
