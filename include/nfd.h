@@ -87,7 +87,10 @@ typedef struct {
 /* Create a context.  `cuda_stream` is a cudaStream_t (NULL = legacy default
  * stream).  Validates cfg (NFD_E_BADCFG), copies/repacks the weights, allocates
  * the cache: n_streams x n_layers x (W + 2 k_max) frame pages of K and of V.
- * Synchronises the stream before returning. */
+ * In bf16 mode the first context of a shape in the process also times its GEMM
+ * tile plans on scratch data (about half a second; the environment variable
+ * NFD_NO_TUNE=1 skips it and keeps the built-in cost model's plans); the cache is
+ * cleared afterwards.  Synchronises the stream before returning. */
 int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cuda_stream);
 int nfd_destroy(nfd_ctx *ctx);
 
