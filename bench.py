@@ -327,7 +327,10 @@ def main():
 
     # ---------------- device-resident leg (the headline `value`) ----------------
     # load-time work, untimed like the weight upload: the modulation table of all (time, action) pairs
-    n_warm = nfd.warm_modulation()
+    try:
+        n_warm = nfd.warm_modulation()
+    except Exception:              # more (time, action) pairs than the table holds: they are computed on demand
+        n_warm = 0
     fill_prompt()
     n_all = K + Wm
     noise = randn(n_all, S, 1, *fs)
