@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *co
 // 32) it also writes the first layer's GEMM operand z*(1+scale) and the row-sum
 // partials of z per 32 columns.
 // ---------------------------------------------------------------------------
-#define PE_TOK 16
+#define PE_TOK 8
 template <typename TS>
 __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
                                                      float *z, TS *a_out, float2 *stats, const float *scale0,
