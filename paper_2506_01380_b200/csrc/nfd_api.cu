@@ -354,11 +354,11 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
     if (c->h_sp.nc > 0) enqueue_conditioning<TS>(c, nf);
     // tokens
     c->cls = CLS_PATCH;
-    if (c->bf16_mode && c->fast)
-        PLAUNCH(c, k_rope_table, (M * (D.dh / 2) + 255) / 256, 256, 0, sp, D, (const RopeTab *)c->d_rope, c->rope_cs);
+    // (the tensor-core QKV epilogue reads the rotary table that the patch embedding writes on the side)
     PLAUNCH(c, (k_patch_embed<TS>), dim3((M + PE_TOK - 1) / PE_TOK, (d + 255) / 256), 256, PE_TOK * D.P * sizeof(float), sp, D,
             (const TS *)c->w_pe_io, (const TS *)c->b_pe, c->z, fold ? (TS *)c->hbuf : (TS *)nullptr, c->ln_stats,
-            (const float *)c->mod + d, mod_row);
+            (const float *)c->mod + d, mod_row, (const RopeTab *)c->d_rope,
+            (c->bf16_mode && c->fast) ? c->rope_cs : (float2 *)nullptr);
     const int ln_grid = (M + 3) / 4;
     for (int l = 0; l < L; ++l) {
         const float *modl = c->mod + (size_t)l * 6 * d;

@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(256) k_modw(const StepParams *sp, const TS *co
 template <typename TS>
 __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims D, const TS *W_pe, const TS *b_pe,
                                                      float *z, TS *a_out, float2 *stats, const float *scale0,
-                                                     size_t mod_row_stride) {
+                                                     size_t mod_row_stride, const RopeTab *rt, float2 *rope_tab) {
     extern __shared__ float s_patch[];          // [PE_TOK][P]
     NFD_TRACE_T0();
     pdl_wait();
@@ -235,6 +235,21 @@ __global__ void __launch_bounds__(256) k_patch_embed(const StepParams *sp, Dims 
     const int M = sp->nf * D.T;
     const int m0 = blockIdx.x * PE_TOK;
     if (m0 >= M) return;
+    if (rope_tab && blockIdx.y == 0) {
+        // the per-pass rotary table (cos, sin) of this CTA's tokens: [token][pair of the head dimension]
+        const int half = D.dh >> 1;
+        for (int idx = threadIdx.x; idx < PE_TOK * half; idx += blockDim.x) {
+            const int m = m0 + idx / half, pi = idx % half;
+            if (m < M) {
+                const int tok = m % D.T;
+                const int ax = rt->axis[pi];
+                const float pos = (float)(ax == 0 ? sp->fr[m / D.T].frame : (ax == 1 ? tok / D.tw : tok % D.tw));
+                float sn, cs;
+                sincosf(pos * rt->freq[pi], &sn, &cs);
+                rope_tab[(size_t)m * half + pi] = make_float2(cs, sn);
+            }
+        }
+    }
     for (int i = threadIdx.x; i < PE_TOK * D.P; i += blockDim.x) {
         const int t = i / D.P, p = i - t * D.P, m = m0 + t;
         float v = 0.f;
@@ -393,25 +408,6 @@ __global__ void __launch_bounds__(128) k_adaln(const StepParams *sp, Dims D, con
                    fmaf((v.y - mean) * rstd, 1.0f + b.y, a.y), fmaf((v.z - mean) * rstd, 1.0f + b.z, a.z),
                    fmaf((v.w - mean) * rstd, 1.0f + b.w, a.w));
     }
-}
-
-// ---------------------------------------------------------------------------
-// Per-pass RoPE table: (cos, sin) of every token's rotation angle for every
-// pair of the head dimension, [nf*T][dh/2].
-// ---------------------------------------------------------------------------
-__global__ void k_rope_table(const StepParams *sp, Dims D, const RopeTab *rt, float2 *tab) {
-    pdl_wait();
-    pdl_launch();
-    const int half = D.dh >> 1;
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= sp->nf * D.T * half) return;
-    const int m = i / half, pi = i % half;
-    const int tok = m % D.T;
-    const int ax = rt->axis[pi];
-    const float pos = (float)(ax == 0 ? sp->fr[m / D.T].frame : (ax == 1 ? tok / D.tw : tok % D.tw));
-    float sn, cs;
-    sincosf(pos * rt->freq[pi], &sn, &cs);
-    tab[i] = make_float2(cs, sn);
 }
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4 &u, float *f) {
