@@ -94,3 +94,64 @@ def test_k1_speculation_is_plain_generation():
     for l in range(cfg["n_layers"]):
         np.testing.assert_allclose(a.kv_frame(l, 0)[0], b.kv_frame(l, 0)[0], atol=1e-12)
         np.testing.assert_allclose(a.kv_frame(l, 0)[1], b.kv_frame(l, 0)[1], atol=1e-12)
+
+
+# ---------------------------------------------------------------- the undistilled sampler's wrapper
+def test_dpmpp_wrapper_equals_the_solver_driven_by_hand():
+    """NFDOracle.sample_dpmpp (Section 3.2 "Sampling") against a twin oracle on which the steps are taken one
+    by one: the model is evaluated on the unit-variance state at the grid's times, the data prediction is
+    x - t v, the solver's result is scaled by sigma_d, and the k frames are committed as tentative."""
+    cfg = micro_cfg()
+    w = I.make_weights(cfg, 5, "stress")
+    a, b = O.NFDOracle(cfg, w), O.NFDOracle(cfg, w)
+    prompt = I.make_latents(cfg, 2, 9).astype(float)
+    for o in (a, b):
+        o.commit_frame(prompt, [0, 1], None)
+    k, n_evals, act = 2, 6, 1
+    nz = np.concatenate([I.make_latents(cfg, 1, 400 + j) for j in range(k)]).astype(float)
+    cz = ctx_noise_for(cfg, 2, k).astype(float)
+    x0 = a.sample_dpmpp(k, act, nz, n_evals=n_evals, ctx_noise=cz)
+    assert (a.n_committed, a.n_tentative) == (2, k)
+    # by hand on the twin: every evaluation is a plain denoise_step on top of the two committed frames
+    seen = []
+
+    def x0_fn(x, t):
+        seen.append(t)
+        assert (b.n_committed, b.n_tentative) == (2, 0)
+        return x - t * b.denoise_step(x, t, act)
+
+    est = cfg["sigma_d"] * O.dpmpp_2m(x0_fn, nz, n_evals)
+    assert seen == O.dpmpp_grid(n_evals)[:-1]
+    np.testing.assert_allclose(x0, est, atol=1e-12)
+    b.commit_frame(est, [act] * k, cz)            # same pages, counted as committed instead of tentative
+    for l in range(cfg["n_layers"]):
+        for f in (2, 3):
+            np.testing.assert_allclose(a.kv_frame(l, f)[0], b.kv_frame(l, f)[0], atol=1e-12)
+            np.testing.assert_allclose(a.kv_frame(l, f)[1], b.kv_frame(l, f)[1], atol=1e-12)
+    a.rollback(1)
+    assert (a.n_committed, a.n_tentative) == (3, 0) and 3 not in a.kv[0]
+
+
+def test_dpmpp_wrapper_closed_form_for_a_constant_velocity():
+    """With every gate of the blocks and the output matrix set to zero the velocity is the output bias b,
+    whatever the input: the probability-flow path is the straight line x(t) = x(1) - (1 - t) b, the data
+    prediction x - t v is the constant x(1) - b along it, and a data-prediction solver returns exactly that.
+    So the generated frame is sigma_d (noise - b): this fixes the sign of x0 = x - t v, that the start is the
+    unit-variance noise itself and that the result is scaled by sigma_d once."""
+    cfg = micro_cfg()
+    w = I.make_weights(cfg, 6, "stress")
+    d = cfg["d_model"]
+    for l in range(cfg["n_layers"]):
+        w[f"w_mod.{l}"][:, 2 * d:3 * d] = 0.0
+        w[f"w_mod.{l}"][:, 5 * d:6 * d] = 0.0
+        w[f"b_mod.{l}"][2 * d:3 * d] = 0.0
+        w[f"b_mod.{l}"][5 * d:6 * d] = 0.0
+    w["w_out"][:] = 0.0
+    o = O.NFDOracle(cfg, w)
+    nz = I.make_latents(cfg, 1, 31).astype(float)
+    # b_out per patch element, laid out as a latent frame (patch = 1 here: one channel vector per token)
+    b_frame = o.unpatchify(np.tile(np.asarray(w["b_out"], float), (o.T, 1)))
+    for n_evals in (1, 3, 18):
+        o.reset()
+        x0 = o.sample_dpmpp(1, 0, nz, n_evals=n_evals)
+        np.testing.assert_allclose(x0, cfg["sigma_d"] * (nz - b_frame), atol=1e-12)
