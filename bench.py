@@ -2,6 +2,7 @@
 """Benchmark of the NFD hot path (libnfd) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --profile-case [...]      (a small self-ending workload for profiler captures)
 
 A "step" generates ONE frame of the 310M-class configuration at batch 1 with a
 16-frame KV context: 4 denoising passes (sampler glue included) plus the commit
@@ -136,9 +137,15 @@ class ClockSampler:
 # ---------------------------------------------------------------------------
 # algorithmic work of one launch of each kernel class (k = 1 pass, steady state)
 # ---------------------------------------------------------------------------
-def class_work(cfg, T, n_ctx):
+def class_work(cfg, T, n_ctx, n_frames=1, n_streams=1):
+    """Algorithmic FLOPs and HBM bytes of one launch of each kernel class in a pass of n_streams x n_frames
+    frames: operands read once, results written once.  Frame j of a stream's chunk sees the n_ctx cached
+    frames, the chunk frames before it and itself."""
     d, dm, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
-    M, Nk = T, (n_ctx + 1) * T
+    nf = n_frames * n_streams
+    M = nf * T
+    keys_per_stream = sum((n_ctx + 1 + j) * T for j in range(n_frames))      # summed over the chunk's frames
+    kv_rows = n_streams * (n_ctx + n_frames) * T                              # distinct K (and V) rows read
 
     def gemm(N, K, res=False):
         return dict(flops=2.0 * M * N * K, bytes=2.0 * (N * K + M * K + M * N) + (8.0 * M * N if res else 0.0))
@@ -148,25 +155,54 @@ def class_work(cfg, T, n_ctx):
         "gemm_out_gate_res": gemm(d, d, True),
         "gemm_fc1_gelu": gemm(n1, d),
         "gemm_fc2_gate_res": gemm(d, dm, True),
-        "attention": dict(flops=4.0 * M * Nk * d, bytes=2.0 * (2 * Nk * d + 2 * M * d)),
+        "attention": dict(flops=4.0 * T * keys_per_stream * n_streams * d, bytes=2.0 * (2 * kv_rows * d + 2 * M * d)),
         "adaln_norm": dict(flops=8.0 * M * d, bytes=M * d * 6.0),
-        "conditioning": dict(flops=2.0 * 6 * d * d, bytes=2.0 * 6 * d * d),   # per layer-launch average
     }
 
 
-# DRAM bytes (read + write) of one launch from the ncu captures summarised under profiles/ (same kernels,
-# 2-layer slice of this shape; one launch of a kernel moves the same bytes whatever the layer count).
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    "attention": 24.13e6,               # profiles/ncu_attention_nfd310m_k1.txt
-    "gemm_qkv_rope_kvstore": 31.46e6,   # profiles/ncu_gemm_nfd310m_k1.txt (includes the K/V page prefetch for attention)
-    "gemm_out_gate_res": 12.69e6,
-    "gemm_fc1_gelu": 17.76e6,
-    "gemm_fc2_gate_res": 19.25e6,
-}
+# DRAM bytes (read + write) of one launch come from the ncu summaries under profiles/: a summary that was
+# taken for this purpose carries lines "traffic <kernel class> <bytes per launch>" and one line
+# "source_sha256 <file under csrc/> <digest>" per kernel source it depends on.  The figure is used only while
+# those sources are unchanged; otherwise `traffic` is null.
+PROFILE_FILES = ["ncu_attention_nfd310m_k1.txt", "ncu_gemm_nfd310m_k1.txt"]
 
 
-def roofline_of(cfg, T, n_ctx, prof, pk):
-    work = class_work(cfg, T, n_ctx)
+def _sha256(path):
+    import hashlib
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def traffic_from_profiles():
+    """{kernel class: (DRAM bytes per launch, profile file)} for the summaries whose kernel sources still match."""
+    out = {}
+    csrc = os.path.join(ROOT, "paper_2506_01380_b200", "csrc")
+    for name in PROFILE_FILES:
+        path = os.path.join(ROOT, "profiles", name)
+        if not os.path.exists(path):
+            continue
+        traffic, fresh, n_sha = {}, True, 0
+        for ln in open(path):
+            w = ln.split()
+            if len(w) == 3 and w[0] == "traffic":
+                traffic[w[1]] = float(w[2])
+            if len(w) == 3 and w[0] == "source_sha256":
+                n_sha += 1
+                src = os.path.join(csrc, w[1])
+                fresh = fresh and os.path.exists(src) and _sha256(src) == w[2]
+        if fresh and n_sha:
+            for k, v in traffic.items():
+                out[k] = (v, "profiles/" + name)
+    return out
+
+
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def roofline_of(cfg, T, n_ctx, prof, pk, n_frames=1, n_streams=1, traffic=None):
+    """Roofline entry of the kernel class with the largest share of `prof` (per-class launches and summed time
+    of passes that all carry n_streams x n_frames frames), each kernel timed by events around its launch."""
+    work = class_work(cfg, T, n_ctx, n_frames, n_streams)
     total = sum(ms for _, ms in prof.values()) or 1.0
     shares = {k: round(ms / total, 4) for k, (n, ms) in prof.items() if n}
     cand = [(ms, k) for k, (n, ms) in prof.items() if n and k in work]
@@ -176,21 +212,24 @@ def roofline_of(cfg, T, n_ctx, prof, pk):
     n = prof[name][0]
     dur = ms / n * 1e-3
     w = work[name]
-    t_flop, t_byte = w["flops"] / (pk["tf_sust"] * 1e12), w["bytes"] / (pk["hbm"] * 1e9)
-    if name == "conditioning":
-        # one class covers several small GEMV launches; report the modulation GEMV bytes of a pass
-        w = dict(flops=0.0, bytes=2.0 * 6 * cfg["d_model"] ** 2 * cfg["n_layers"])
-        dur = ms / (n / 5.0) * 1e-3
-        t_flop, t_byte = 0.0, 1.0
+    # a kernel timed alone between two events: the burst figures are the denominators
+    t_flop, t_byte = w["flops"] / (pk["tf_burst"] * 1e12), w["bytes"] / (pk["hbm"] * 1e9)
     if t_flop >= t_byte:
-        ach, peak, unit, bound = w["flops"] / dur / 1e12, pk["tf_sust"], "TFLOP/s", "tensor"
+        ach, peak, unit, bound = w["flops"] / dur / 1e12, pk["tf_burst"], "TFLOP/s", "tensor"
     else:
         ach, peak, unit, bound = w["bytes"] / dur / 1e9, pk["hbm"], "GB/s", "hbm"
-    return {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
-            "frac": round(ach / peak, 4), "peak_source": pk["src"] + (" (sustained)" if bound == "tensor" else ""),
-            "avg_launch_us": round(dur * 1e6, 2), "share_of_step": shares.get(name),
-            "algorithmic_bytes": w["bytes"], "algorithmic_flops": w["flops"],
-            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(name)}, shares
+    r = {"kernel": name, "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
+         "frac": round(ach / peak, 4),
+         "peak_source": pk["src"] + (" (bf16 burst: kernel timed alone)" if bound == "tensor" else " (copy)"),
+         "avg_launch_us": round(dur * 1e6, 2), "launches_timed": n, "frames_per_pass": n_frames * n_streams,
+         "share_of_step": shares.get(name),
+         "algorithmic_bytes": w["bytes"], "algorithmic_flops": w["flops"], "traffic": None}
+    if bound == "tensor":
+        r["frac_of_measured_sustained"] = round(ach / pk["tf_sust"], 4)
+        r["frac_of_nominal_bf16_dense"] = round(ach / NOMINAL_BF16_TFLOPS, 4)
+    if traffic and name in traffic and n_frames == 1 and n_streams == 1:
+        r["traffic"], r["traffic_source"] = traffic[name]
+    return r, shares
 
 
 # ---------------------------------------------------------------------------
@@ -230,7 +269,10 @@ def cpu_threads():
 
 
 def run_reference(args):
-    """Reference arm = the oracle on the host cores (the paper ships no code)."""
+    """Reference arm = the oracle on the host cores (the paper ships no code).  A step of this arm is ONE
+    forward pass (k = 1 behind a full context): a whole frame is n_steps + 1 of them and would take most of a
+    minute, so `ms_per_step` is the time of a pass, which is what was timed, and `value` is extrapolated from
+    it to frames/s."""
     from paper_2506_01380_b200 import inputs as I
     import numpy  # noqa: F401  (loads BLAS so that the thread count is known)
     wl_cfg, wl_over, wl_text = WORKLOADS[args.workload]
@@ -241,18 +283,64 @@ def run_reference(args):
     t_pass = sum(times) / len(times)
     passes_per_frame = cfg["n_steps"] + 1
     value = 1.0 / (passes_per_frame * t_pass)
-    sample = (f"each step = 1 forward pass (k=1, 16-frame context of random K/V pages); a frame = "
-              f"{passes_per_frame} passes, value extrapolated as 1/({passes_per_frame}*t_pass); "
-              f"steps capped at {steps}")
+    sample = (f"a step of this arm = 1 forward pass (k=1, 16-frame context of random K/V pages), {steps} of them "
+              f"timed after {warm} warm-up (the request was capped at 6 steps, 1 warm-up); ms_per_step is the "
+              f"time of a pass; a frame = {passes_per_frame} passes, value extrapolated as "
+              f"1/({passes_per_frame} * t_pass)")
     line = {"impl": "reference", "metric": metric_name(args.workload), "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": steps, "warmup": warm, "ms_per_step": t_pass * passes_per_frame * 1e3,
+            "steps": steps, "warmup": warm, "ms_per_step": t_pass * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl_text},
+            "data": "synthetic", "config": {"workload": wl_text, "step": "one forward pass (see cpu_baseline.sample)"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+def profile_case(argv):
+    """Small, self-ending workload for profiler captures of the library's kernels:
+
+        python bench.py --profile-case [--layers 2] [--ctx 16] [--k 1] [--passes 2] [--no-graph] [--no-fast]
+                                       [--no-prefetch]
+
+    The 310M-class shape with few layers (well under a GB on the device), the KV context filled by commit
+    passes, then a few denoising passes.  Meant to be wrapped by `ncu -k regex:... -c N`."""
+    import torch
+    from paper_2506_01380_b200 import inputs as I
+    from paper_2506_01380_b200.nfd import NFD
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--profile-case", action="store_true")
+    ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--ctx", type=int, default=16)
+    ap.add_argument("--k", type=int, default=1)
+    ap.add_argument("--passes", type=int, default=2)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-fast", action="store_true")
+    ap.add_argument("--no-prefetch", action="store_true")
+    a = ap.parse_args(argv)
+    cfg = I.make_cfg("nfd310m", n_layers=a.layers, ctx_frames=a.ctx)
+    dev = torch.device("cuda:0")
+    nfd = NFD(cfg, torch_weights(cfg, dev, seed=0))
+    if a.no_graph:
+        nfd.set_option("graph", 0)
+    if a.no_fast:
+        nfd.set_option("fast", 0)
+    if a.no_prefetch:
+        nfd.set_option("l2_prefetch", 0)
+    g = torch.Generator(device=dev)
+    g.manual_seed(0)
+    fs = I.frame_shape(cfg)
+    for i in range(0, a.ctx, 4):
+        n = min(4, a.ctx - i)
+        nfd.commit_frame(torch.randn((n,) + fs, generator=g, device=dev), [1] * n)
+    x = torch.randn((a.k,) + fs, generator=g, device=dev)
+    for _ in range(a.passes):
+        v = nfd.denoise_step(x, 0.7, 3)
+    torch.cuda.synchronize()
+    assert nfd.status() == 0
+    print("ok", float(v.abs().mean()))
+    return 0
 
 
 def torch_weights(cfg, device, seed):
@@ -277,10 +365,15 @@ def main():
                          "size-table shapes with a gated MLP (second workload, same step definition)")
     ap.add_argument("--dpmpp", action="store_true",
                     help="add the undistilled sampler leg (DPM-Solver++, 18 function evaluations per frame)")
-    ap.add_argument("--batch8", action="store_true",
-                    help="add the 8-stream, 32-frame-context leg (aggregate and per-stream frames/s)")
+    ap.add_argument("--no-batch8", action="store_true",
+                    help="skip the 8-stream, 32-frame-context leg (aggregate and per-stream frames/s)")
     ap.add_argument("--spec-sweep", action="store_true",
                     help="add accepted frames/s for k = 1..4 over action chains of several repeat probabilities")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="repeat the timed region of --steps frames until this much time was timed in all; the "
+                         "reported value is the median region")
+    if "--profile-case" in sys.argv[1:]:
+        return profile_case(sys.argv[1:])
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -337,6 +430,20 @@ def main():
     cnoise = randn(n_all, 1, *fs)
     actions = I.make_actions_uniform(cfg, n_all, rank)
     x0 = torch.empty((1,) + fs, device=device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_region():
+        """EXACTLY K steps between two events on the library's stream, a barrier and a device synchronise on
+        both sides; returns the slowest rank's milliseconds."""
+        barrier()
+        e0.record(nfd.stream)
+        for i in range(Wm, n_all):
+            nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
+            nfd.rollback(1)
+        e1.record(nfd.stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1), dist, device)
+
     with torch.cuda.stream(nfd.stream):
         for i in range(Wm):
             nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
@@ -345,16 +452,15 @@ def main():
         clocks = ClockSampler(device)
         clocks.start()
         l0 = nfd.launch_count()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(nfd.stream)
-        for i in range(Wm, n_all):
-            nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
-            nfd.rollback(1)
-        e1.record(nfd.stream)
-        barrier()
-        clk = clocks.stop()
-        ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
+        regions = [timed_region()]
         launches = nfd.launch_count() - l0
+        # short regions are repeated (same K steps each, the stream just goes on generating) until at least
+        # --min-seconds were timed; every rank takes the same number of regions
+        n_rep = int(min(64, max(1, math.ceil(args.min_seconds * 1e3 / max(regions[0], 1e-3)))))
+        for _ in range(n_rep - 1):
+            regions.append(timed_region())
+        clk = clocks.stop()
+        ms = sorted(regions)[len(regions) // 2]
     assert nfd.status() == 0
     hits, misses = nfd.cond_cache_stats()
     value = aggregate_frames_per_s(world, K, ms)
@@ -363,6 +469,8 @@ def main():
             "warmup": Wm,
             "ms_per_step": round(ms / K, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
+            "timed_regions": {"count": len(regions), "steps_each": K, "reported": "median",
+                              "ms_each": [round(r, 3) for r in regions], "ms_total": round(sum(regions), 2)},
             "config": {"workload": wl_text, "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2: the weights (604 MB for nfd310m) and the KV pages (528 MB) are "
                              "streamed every pass",
@@ -379,7 +487,7 @@ def main():
                                          "activation and timed extent not stated: context, not a baseline"}
     if rank == 0 and world == 1 and not args.no_extras:
         # ---------------- end-to-end leg: host buffers in, host frame out ----------------
-        n_e = min(K, 32)
+        n_e = max(8, min(K, 32))
         h_noise = torch.randn(n_e, S, 1, *fs).pin_memory()
         h_cn = torch.randn(n_e, 1, *fs).pin_memory()
         h_out = torch.empty((1,) + fs).pin_memory()
@@ -390,7 +498,7 @@ def main():
             for i in range(n_e):
                 d_noise.copy_(h_noise[i], non_blocking=True)
                 d_cn.copy_(h_cn[i], non_blocking=True)
-                nfd.speculate(1, actions[i], d_noise, d_cn, out=x0)
+                nfd.speculate(1, actions[i % n_all], d_noise, d_cn, out=x0)
                 nfd.rollback(1)
                 h_out.copy_(x0, non_blocking=True)
                 nfd.stream.synchronize()          # the caller needs the frame before choosing the next action
@@ -453,45 +561,6 @@ def main():
                                "n_evals": 18, "forward_passes_per_frame": 19, "steps": n_d,
                                "paper_context_fps_a100": {"nfd310m": 6.15}.get(args.workload)}
 
-        # ---------------- 8 independent streams, 32-frame context, one batched call per frame ----------------
-        if args.batch8:
-            nb = 8
-            cfg8 = dict(cfg, ctx_frames=32, n_streams=nb)
-            nfd.close()
-            nfd8 = NFD(cfg8, torch_weights(cfg8, device, seed=0), device=str(device))
-            nfd8.warm_modulation()
-            streams = list(range(nb))
-            for st in streams:
-                acts = I.make_actions_uniform(cfg8, 32, 100 + st)
-                for i in range(0, 32, 4):
-                    nfd8.commit_frame(randn(4, *fs), acts[i:i + 4], randn(4, *fs), stream=st)
-            n8 = 16
-            acts8 = [I.make_actions_uniform(cfg8, n8 + 3, st) for st in streams]
-            nz8, cz8 = randn(S, nb, 1, *fs), randn(nb, 1, *fs)
-            x8 = torch.empty((nb, 1) + fs, device=device)
-            with torch.cuda.stream(nfd8.stream):
-                for i in range(3):
-                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
-                    for st in streams:
-                        nfd8.rollback(1, stream=st)
-                torch.cuda.synchronize(device)
-                e0.record(nfd8.stream)
-                for i in range(3, n8 + 3):
-                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
-                    for st in streams:
-                        nfd8.rollback(1, stream=st)
-                e1.record(nfd8.stream)
-                torch.cuda.synchronize(device)
-            assert nfd8.status() == 0
-            ms8 = e0.elapsed_time(e1)
-            line["batch8_ctx32"] = {"aggregate_frames_per_s": round(nb * n8 / (ms8 * 1e-3), 2),
-                                    "per_stream_frames_per_s": round(n8 / (ms8 * 1e-3), 2),
-                                    "ms_per_batched_frame_step": round(ms8 / n8, 3), "streams": nb, "ctx_frames": 32,
-                                    "steps": n8}
-            nfd8.close()
-            nfd = NFD(cfg, torch_weights(cfg, device, seed=0), device=str(device))
-            nfd.warm_modulation()
-
         # ---------------- speculation depth x action repeat probability ----------------
         if args.spec_sweep:
             rows = []
@@ -525,19 +594,48 @@ def main():
                                  "ms_per_speculate": round(ms_k / passes, 3)})
             line["spec_sweep"] = rows
 
-        # ---------------- per-kernel timing (events around every launch) ----------------
+        # ---------------- per-kernel timing (events around every launch, graph off) ----------------
+        # Teacher-forced passes behind the full 16-frame context, so that every launch of a class does the same
+        # work: passes of one frame (three of the four launched passes of a steady-state step) and passes of
+        # two frames (the fourth, which carries the previous frame's commit).
+        traffic = traffic_from_profiles()
         fill_prompt()
+        xt1, xt2 = randn(1, *fs), randn(2, *fs)
         with torch.cuda.stream(nfd.stream):
+            nfd.denoise_step(xt1, 0.7, 3)
             nfd.profile_begin()
-            for i in range(4):
+            for _ in range(6):
+                nfd.denoise_step(xt1, 0.7, 3)
+            prof1 = nfd.profile_end()
+            nfd.denoise_step(xt2, 0.7, 3)
+            nfd.profile_begin()
+            for _ in range(4):
+                nfd.denoise_step(xt2, 0.7, 3)
+            prof2 = nfd.profile_end()
+            # shares over a whole steady-state step, as the bench's timed loop runs it
+            fill_prompt()
+            nfd.speculate(1, actions[0], noise[0], cnoise[0], out=x0)
+            nfd.rollback(1)
+            nfd.profile_begin()
+            for i in range(1, 4):
                 nfd.speculate(1, actions[i], noise[i], cnoise[i], out=x0)
                 nfd.rollback(1)
             prof = nfd.profile_end()
-        roof, shares = roofline_of(cfg, T, W, prof, pk)
+        roof, _ = roofline_of(cfg, T, W, prof1, pk, n_frames=1, traffic=traffic)
+        roof2, _ = roofline_of(cfg, T, W, prof2, pk, n_frames=2)
+        total = sum(ms_ for _, ms_ in prof.values()) or 1.0
+        shares = {k_: round(ms_ / total, 4) for k_, (n_, ms_) in prof.items() if n_}
+        if roof:
+            roof["share_of_step"] = shares.get(roof["kernel"])
         if roof and args.workload != "nfd310m":
             roof["traffic"] = None           # the ncu captures are of the nfd310m shape
         line["roofline"] = roof
+        line["roofline_two_frame_pass"] = roof2
         line["kernel_time_shares"] = shares
+        line["per_launch_us"] = {
+            "one_frame_pass": {k_: round(ms_ / n_ * 1e3, 2) for k_, (n_, ms_) in prof1.items() if n_},
+            "two_frame_pass": {k_: round(ms_ / n_ * 1e3, 2) for k_, (n_, ms_) in prof2.items() if n_},
+            "note": "CUDA events around every launch, graph off: launch latency is inside each figure"}
         # whole-pass roofline: the slower of FLOPs at the bf16 peak and bytes at HBM bandwidth
         d, dm, L = cfg["d_model"], cfg["d_mlp"], cfg["n_layers"]
         gemm_params = L * (4 * d * d + (3 if cfg.get("act", 0) == 1 else 2) * d * dm)
@@ -546,7 +644,68 @@ def main():
         t_roof = max(flops / (pk["tf_sust"] * 1e12), byts / (pk["hbm"] * 1e9))
         line["pass_roofline"] = {"flops_per_pass": flops, "bytes_per_pass": byts,
                                  "roofline_frames_per_s": round(1.0 / ((S + 1) * t_roof), 1),
-                                 "frac": round(value / (1.0 / ((S + 1) * t_roof)), 4), "peak_source": pk["src"]}
+                                 "frac": round(value / (1.0 / ((S + 1) * t_roof)), 4),
+                                 "peak_source": pk["src"] + " (sustained bf16: the pass is timed inside a long loop; "
+                                                            "copy bandwidth)"}
+
+        # ---------------- 8 independent streams, 32-frame context, one batched call per frame ----------------
+        if not args.no_batch8 and args.workload == "nfd310m":
+            nb = 8
+            cfg8 = dict(cfg, ctx_frames=32, n_streams=nb)
+            nfd.close()
+            nfd8 = NFD(cfg8, torch_weights(cfg8, device, seed=0), device=str(device))
+            nfd8.warm_modulation()
+            streams = list(range(nb))
+
+            def fill8():
+                for st in streams:
+                    nfd8.reset(st)
+                    acts = I.make_actions_uniform(cfg8, 32, 100 + st)
+                    for i in range(0, 32, 4):
+                        nfd8.commit_frame(randn(4, *fs), acts[i:i + 4], randn(4, *fs), stream=st)
+            fill8()
+            n8 = 16
+            acts8 = [I.make_actions_uniform(cfg8, n8 + 3, st) for st in streams]
+            nz8, cz8 = randn(S, nb, 1, *fs), randn(nb, 1, *fs)
+            x8 = torch.empty((nb, 1) + fs, device=device)
+            with torch.cuda.stream(nfd8.stream):
+                for i in range(3):
+                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
+                    for st in streams:
+                        nfd8.rollback(1, stream=st)
+                torch.cuda.synchronize(device)
+                e0.record(nfd8.stream)
+                for i in range(3, n8 + 3):
+                    nfd8.speculate_batched(streams, 1, [int(a[i]) for a in acts8], nz8, cz8, out=x8)
+                    for st in streams:
+                        nfd8.rollback(1, stream=st)
+                e1.record(nfd8.stream)
+                torch.cuda.synchronize(device)
+            assert nfd8.status() == 0
+            ms8 = e0.elapsed_time(e1)
+            b8 = {"aggregate_frames_per_s": round(nb * n8 / (ms8 * 1e-3), 2),
+                  "per_stream_frames_per_s": round(n8 / (ms8 * 1e-3), 2),
+                  "ms_per_batched_frame_step": round(ms8 / n8, 3), "streams": nb, "ctx_frames": 32, "steps": n8,
+                  "workload": "BASELINE config 5: 8 independent streams, 32-frame KV context, 4 steps + commit"}
+            # its dominant kernel: teacher-forced batched passes of 8 x 1 frames behind the full contexts
+            fill8()
+            xt8 = randn(nb, 1, *fs)
+            with torch.cuda.stream(nfd8.stream):
+                nfd8.denoise_step_batched(streams, xt8, [0.7] * nb, [3] * nb)
+                nfd8.profile_begin()
+                for _ in range(3):
+                    nfd8.denoise_step_batched(streams, xt8, [0.7] * nb, [3] * nb)
+                prof8 = nfd8.profile_end()
+            b8["roofline"], b8["kernel_time_shares"] = roofline_of(cfg8, T, 32, prof8, pk, n_frames=1, n_streams=nb)
+            f8 = 2.0 * nb * T * gemm_params + 4.0 * nb * T * 33 * T * d * L
+            y8 = 2.0 * gemm_params + 2.0 * 2 * L * 32 * T * d * nb
+            t8 = max(f8 / (pk["tf_sust"] * 1e12), y8 / (pk["hbm"] * 1e9))
+            b8["pass_roofline"] = {"flops_per_pass": f8, "bytes_per_pass": y8,
+                                   "roofline_aggregate_frames_per_s": round(nb / ((S + 1) * t8), 1),
+                                   "frac": round(b8["aggregate_frames_per_s"] / (nb / ((S + 1) * t8)), 4),
+                                   "peak_source": pk["src"] + " (sustained bf16, copy bandwidth)"}
+            line["batch8_ctx32"] = b8
+            nfd8.close()
 
         # ---------------- the oracle on this machine's host cores ----------------
         t_or = oracle_sample(cfg, 2)

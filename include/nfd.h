@@ -90,7 +90,14 @@ typedef struct {
  * In bf16 mode the first context of a shape in the process also times its GEMM
  * tile plans on scratch data (about half a second; the environment variable
  * NFD_NO_TUNE=1 skips it and keeps the built-in cost model's plans); the cache is
- * cleared afterwards.  Synchronises the stream before returning. */
+ * cleared afterwards.  The plan found fixes, among other things, over how many
+ * thread blocks the K range of a projection is split, hence the order in which
+ * its products are summed: all contexts of one process share the plans and give
+ * bitwise equal results for equal inputs, two processes may differ in the last
+ * bits (NFD_NO_TUNE=1 makes the plans, and with them the bits, the same
+ * everywhere).  A bf16 context needs the driver's cuTensorMapEncodeTiled entry
+ * point; without it the call fails with NFD_E_CUDA rather than run the plain
+ * validation kernels unasked.  Synchronises the stream before returning. */
 int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cuda_stream);
 int nfd_destroy(nfd_ctx *ctx);
 
@@ -138,9 +145,8 @@ int nfd_commit_frame(nfd_ctx *ctx, int stream, const float *x0, int n, const int
  * The K/V pages of the k frames are not written by this call: the library keeps
  * a copy of the clean frames, their context noise and the action, counts the
  * frames as tentative, and lets them ride along (K/V only) in the first
- * denoising pass of the next nfd_speculate on this batch slot -- the paper's
- * "compute and cache their KVs during the first denoising step" (Appendix,
- * KV caching).  Any call that needs the pages earlier (nfd_kv_hash,
+ * denoising pass of the next nfd_speculate on this batch slot, which is where
+ * the paper's appendix on KV caching places that computation.  Any call that needs the pages earlier (nfd_kv_hash,
  * nfd_kv_read, nfd_denoise_step*, nfd_commit_frame) writes them first.  Results
  * are bitwise those of committing at once (option "lazy_commit" = 0). */
 int nfd_speculate(nfd_ctx *ctx, int stream, int k, int action, const float *noise, const float *ctx_noise,
@@ -216,8 +222,33 @@ int nfd_attention_noalloc(const void *q, const void *k_pages, const void *v_page
                           void *out, void *cuda_stream);
 
 /* Device-side status latch: 0, or the first NFD_E_* a kernel recorded.
- * Synchronises the stream. */
+ * NFD_E_TIMEOUT: a bounded wait inside a kernel (on an mbarrier that a TMA copy or
+ * a tensor-core operation completes) ran out after 0.4 s; the kernel skipped the
+ * rest of its work and left by its normal exit, so the context still runs, but
+ * the results of that pass are void.  NFD_E_DEVICE: the first kernel of a pass
+ * found an index in the pass descriptor outside the context's limits (batch slot,
+ * window, modulation row, frame slots); the frames of that pass were redirected
+ * to batch slot 0 so that no kernel left its buffers: treat every cache of the
+ * context as lost (nfd_reset).  The latch keeps the first code until
+ * nfd_set_option("clear_status", 1).  Synchronises the stream. */
 int nfd_status(nfd_ctx *ctx);
+
+/* Verification of a speculation (Section 4.2 and the control flow of the
+ * appendix listing): frames i .. i+k-1 were generated under actions[i]
+ * (host array of the n true actions).  Returns how many leading frames were
+ * generated under their own true action -- at least 1, at most k and n - i --
+ * which is the n_accept to pass to nfd_rollback; or a negative code. */
+int nfd_accepted_count(const int *actions, int n, int i, int k);
+
+/* Copy the first n_elems elements of one activation buffer of the last pass to
+ * dev fp32 memory, for kernel-level tests: "z" the residual stream [rows, d]
+ * (fp32), "hbuf" the operand of the QKV / first MLP projection [rows, d], "qbuf"
+ * the rotated queries [n_heads, rows, head_dim], "abuf" the attention output
+ * [rows, d], "mbuf" the MLP hidden activation [rows, d_mlp rounded up to a
+ * multiple of 8].  rows = frames of the pass x T.  Buffers are reused by every
+ * layer, so what is read belongs to the last layer that wrote it.
+ * NFD_E_RANGE for another name or more elements than the buffer holds. */
+int nfd_debug_read(nfd_ctx *ctx, const char *name, float *out, long long n_elems);
 
 /* Number of kernels the library launched (or replayed inside graphs) since
  * creation. */
@@ -225,7 +256,7 @@ long long nfd_launch_count(nfd_ctx *ctx);
 
 /* The adaLN modulation of a frame (Section 3.1, "Action Conditioning") depends on
  * its (FM time, action) pair only.  The library keeps the modulation of the most
- * recently used pairs (96 of them) and computes a pair's modulation only when it
+ * recently used pairs (256 of them) and computes a pair's modulation only when it
  * is not there.  Returns how many pairs were found (hits) and how many had to be
  * computed (misses) since creation; either pointer may be NULL. */
 int nfd_cond_cache_stats(nfd_ctx *ctx, long long *hits, long long *misses);
@@ -271,8 +302,20 @@ int nfd_warm_modulation(nfd_ctx *ctx);
  * once), "fuse_ln" 0/1 (bf16 tensor-core path: fold the two adaLN LayerNorms of
  * every block into the epilogues of the neighbouring GEMMs, or run them as
  * kernels of their own; the two differ by bf16 rounding of the GEMM operand
- * only).  Changing "fast" or "fuse_ln" empties the modulation cache.  Returns
- * NFD_E_RANGE for unknown names. */
+ * only), "l2_prefetch" 0/1 (each GEMM pulls the next GEMM's weights, the QKV
+ * GEMM also the layer's cached K/V pages, towards L2), "clear_status" (reset the
+ * device-side status latch).  Changing "fast" or "fuse_ln" empties the
+ * modulation cache.
+ * Switches that exist for the tests of the error paths; each makes a fault on
+ * the host or lets a bounded wait expire, none makes the device fault:
+ * "test_fail_launch" 1: the next nfd_speculate's first launch asks for a block
+ * size the runtime refuses, so the call returns NFD_E_CUDA; "test_corrupt_desc"
+ * 1: the next pass descriptor names a batch slot that does not exist, which the
+ * pass's first kernel must catch (NFD_E_DEVICE); "test_skip_stage" 1/0: the TMA
+ * producer of every tensor-core GEMM leaves out its last pipeline stage, so that
+ * the consumer's wait for it expires (NFD_E_TIMEOUT); "test_wait_limit_us" n:
+ * bounded waits give up after n microseconds instead of 0.4 s (0 = default).
+ * Returns NFD_E_RANGE for unknown names. */
 int nfd_set_option(nfd_ctx *ctx, const char *name, int value);
 
 const char *nfd_strerror(int code);

@@ -37,11 +37,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     cmd = [
         _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-        "-shared", "-Xcompiler", "-fPIC", "--use_fast_math=false",
+        "-shared", "-Xcompiler", "-fPIC",
         "-I", os.path.join(ROOT, "include"), "-I", CSRC,
         "-o", LIB,
     ] + [os.path.join(CSRC, s) for s in SOURCES]
-    cmd = [c for c in cmd if c != "--use_fast_math=false"]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -43,7 +43,13 @@ struct nfd_ctx {
     size_t esz = 4;
     bool use_graph = true, fast = true;
     long long launches = 0;
-    cudaError_t launch_err = cudaSuccess;    // first failed launch of the current pass
+    cudaError_t launch_err = cudaSuccess;    // first failed launch since the last take_launch_err()
+    // test switches (nfd_set_option "test_*"): each acts on the next call only
+    bool test_fail_launch = false;           // the next sampler launch gets a block size the runtime refuses
+    bool test_corrupt_desc = false;          // the next pass descriptor names a batch slot that does not exist
+    int test_words[4] = {0, 0, 0, 0};        // host copies of the status block's test words (sources of async copies)
+    bool l2_prefetch = true;                 // GEMMs pull the next GEMM's weights towards L2
+    bool kv_prefetch = false;                // the QKV GEMM pulls the layer's cached K/V pages towards L2
     std::vector<void *> allocs;
 
     // repacked weights: matrices [out][in], storage type
@@ -66,7 +72,8 @@ struct nfd_ctx {
     StepParams *d_sp = nullptr;
     StepParams h_sp;
     unsigned long long *d_hash = nullptr;
-    int *d_status = nullptr;
+    int *d_status = nullptr;                // status block of four ints (see nfd_sm100.cuh)
+    DescLimits lim;
     FastState fs;
 
     std::vector<int> n_committed, n_tentative;
@@ -266,12 +273,22 @@ static void prof_mark(nfd_ctx *c, bool stop) {
         (c)->launches++;                                                                            \
     } while (0)
 
+// The first launch error recorded since the last call of this function; the record is cleared, so that one
+// refused launch fails the call it belongs to and nothing after it.
+static cudaError_t take_launch_err(nfd_ctx *c) {
+    cudaError_t e = c->launch_err;
+    c->launch_err = cudaSuccess;
+    if (e == cudaSuccess) e = cudaGetLastError();
+    else cudaGetLastError();
+    return e;
+}
+
 template <typename TS, typename Epi>
 static void launch_gemm(nfd_ctx *c, const TS *A, const TS *Wt, int M, int N, int K, Epi epi, int tc_kind,
                         const void *next_w = nullptr, size_t next_elems = 0, bool folded = false) {
     prof_mark(c, false);
     // the next GEMM's weights, pulled towards L2 by this launch
-    const L2Prefetch pf{next_w, next_w ? (unsigned long long)(next_elems * sizeof(TS)) & ~15ull : 0ull};
+    const L2Prefetch pf{next_w, next_w && c->l2_prefetch ? (unsigned long long)(next_elems * sizeof(TS)) & ~15ull : 0ull};
     if (fast_gemm<TS, Epi>(c->fast && c->bf16_mode, c->fs, c->st, A, Wt, M, N, K, epi, tc_kind, pf)) {
         prof_mark(c, true);
         c->launches++;
@@ -373,7 +390,7 @@ template <typename TS> static void enqueue_body(nfd_ctx *c, int nf, int kind) {
                     (size_t)0, (size_t)d);
         }
         EpiQKV<TS> eq{sp, (const TS *)c->b_qkv[l], (TS *)c->qbuf, (TS *)c->kc, (TS *)c->vc, c->d_rope, D, l,
-                      c->rope_cs, M, lq};
+                      c->rope_cs, M, lq, c->kv_prefetch ? 1 : 0};
         c->cls = CLS_GEMM_QKV;
         launch_gemm<TS>(c, (const TS *)c->hbuf, (const TS *)c->w_qkv[l], M, 3 * d, d, eq, TC_QKV, c->w_o[l],
                         (size_t)d * d, fold);
@@ -422,7 +439,7 @@ static int tune_gemms(nfd_ctx *c) {
     const Dims &D = c->D;
     const int d = D.d, T = D.T;
     FastState &fs = c->fs;
-    if (!c->bf16_mode || !c->fast || !fs.ready || getenv("NFD_NO_TUNE") || getenv("NFD_GEMM_PLAN")) return NFD_OK;
+    if (!c->bf16_mode || !c->fast || !fs.ready || getenv("NFD_NO_TUNE")) return NFD_OK;
     const bool fold = c->fold_active();
     const size_t mod_row = (size_t)D.L * 6 * d, uv_row = (size_t)D.L * (3 * d + D.n1);
     struct Kind { int tc, N, K; };
@@ -493,7 +510,7 @@ static int tune_gemms(nfd_ctx *c) {
             p.fr[j].stream = 0, p.fr[j].frame = j, p.fr[j].win_first = 0, p.fr[j].cond_row = 0, p.fr[j].first_new = 0;
             p.fr[j].src = 0, p.fr[j].src_index = j, p.fr[j].out_index = -1;
         }
-        k_set_params<<<1, 256, 0, c->st>>>(p, c->d_sp);
+        k_set_params<<<1, 256, 0, c->st>>>(p, c->d_sp, c->lim, c->d_status);
         CK(cudaGetLastError());
         touched = true;
         for (int ki = 0; ki < 4; ++ki) {
@@ -511,8 +528,6 @@ static int tune_gemms(nfd_ctx *c) {
             float t_best = 1e30f;
             GemmPlan best = model;
             if (!time_of(ki, M, model.BN, model.S, &t_best)) t_best = 1e30f;
-            if (getenv("NFD_TUNE_LOG") && nf <= 2)
-                fprintf(stderr, "libnfd:   kind %d M %d model BN %d S %d: %.2f us\n", kk, M, model.BN, model.S, t_best);
             t_best *= 0.97f;
             for (int S = 1; S <= 4; S *= 2) {
                 if (!s_open && S != g_tuned_S[skey]) continue;
@@ -525,16 +540,11 @@ static int tune_gemms(nfd_ctx *c) {
                     if (ctas > 3LL * fs.n_sm) continue;          // hopeless: several waves
                     float t;
                     const bool ok_t = time_of(ki, M, BN, S, &t);
-                    if (getenv("NFD_TUNE_LOG") && nf <= 2)
-                        fprintf(stderr, "libnfd:   kind %d M %d BN %d S %d: %.2f us%s\n", kk, M, BN, S, t, ok_t ? "" : " (failed)");
                     if (ok_t && t < t_best) t_best = t, best = GemmPlan{BN, S};
                 }
             }
             if (s_open) g_tuned_S[skey] = best.S;
             g_tuned_BN[bkey] = best.BN;
-            if (getenv("NFD_TUNE_LOG"))
-                fprintf(stderr, "libnfd: tuned kind %d N %d K %d M %d -> BN %d S %d (model BN %d S %d)\n", kk, k.N, k.K, M,
-                        best.BN, best.S, model.BN, model.S);
         }
     }
     cudaEventDestroy(e0);
@@ -544,7 +554,7 @@ static int tune_gemms(nfd_ctx *c) {
         const size_t cache_bytes = (size_t)D.n_streams * D.L * D.R * D.page_elems * c->esz;
         CK(cudaMemsetAsync(c->kc, 0, cache_bytes, c->st));
         CK(cudaMemsetAsync(c->vc, 0, cache_bytes, c->st));
-        CK(cudaMemsetAsync(c->d_status, 0, 4, c->st));
+        CK(cudaMemsetAsync(c->d_status, 0, 16, c->st));
         CK(cudaStreamSynchronize(c->st));
         memset(&c->h_sp, 0, sizeof(c->h_sp));
     }
@@ -563,6 +573,11 @@ static int run_pass_inner(nfd_ctx *c);
 // Run the pass described by c->h_sp.  If it cannot be enqueued, the cache slots that it was to fill are
 // given up again.
 static int run_pass(nfd_ctx *c) {
+    if (c->test_corrupt_desc) {
+        // test switch: a batch slot that does not exist; the first kernel of the pass must catch it
+        c->test_corrupt_desc = false;
+        c->h_sp.fr[0].stream = c->cfg.n_streams + 7;
+    }
     const int rc = run_pass_inner(c);
     if (rc != NFD_OK)
         for (int r = 0; r < c->h_sp.nc; ++r) c->cond_slots[c->h_sp.cd[r].slot] = nfd_ctx::CondSlot();
@@ -573,26 +588,27 @@ static int run_pass_inner(nfd_ctx *c) {
     const int nf = c->h_sp.nf, kind = c->h_sp.kind;
     if (!c->use_graph || c->st == nullptr || c->prof) {
         c->cls = CLS_PARAMS;
-        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp, c->lim, c->d_status);
         enqueue_body_any(c, nf, kind);
-        CK(cudaGetLastError());
-        CK(c->launch_err);
+        CK(take_launch_err(c));
         return NFD_OK;
     }
-    const int key = kind * 64 + nf + (c->fast ? 0 : 4096) + (c->h_sp.nc > 0 ? 0 : 8192) + (c->fuse_ln ? 0 : 16384);   // no conditioning kernels when all pairs are cached
+    // (no conditioning kernels when all pairs are cached)
+    const int key = kind * 64 + nf + (c->fast ? 0 : 4096) + (c->h_sp.nc > 0 ? 0 : 8192) + (c->fuse_ln ? 0 : 16384) +
+                    (c->l2_prefetch ? 0 : 32768) + (c->kv_prefetch ? 0 : 65536);
     auto it = c->graphs.find(key);
     if (it == c->graphs.end()) {
         GraphEntry ge;
         long long before = c->launches;
         CK(cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal));
-        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp, c->lim, c->d_status);
         enqueue_body_any(c, nf, kind);
         cudaError_t e = cudaStreamEndCapture(c->st, &ge.graph);
         ge.launches = c->launches - before;
         c->launches = before;
-        if (e == cudaSuccess && c->launch_err != cudaSuccess) e = c->launch_err;
+        const cudaError_t le = take_launch_err(c);
+        if (e == cudaSuccess) e = le;
         if (e != cudaSuccess || !ge.graph) {
-            c->launch_err = cudaSuccess;
             fprintf(stderr, "libnfd: graph capture failed: %s\n", cudaGetErrorString(e));
             cudaGetLastError();
             return NFD_E_CUDA;
@@ -609,7 +625,7 @@ static int run_pass_inner(nfd_ctx *c) {
         it = c->graphs.emplace(key, ge).first;
     }
     GraphEntry &ge = it->second;
-    void *args[2] = {(void *)&c->h_sp, (void *)&c->d_sp};
+    void *args[4] = {(void *)&c->h_sp, (void *)&c->d_sp, (void *)&c->lim, (void *)&c->d_status};
     cudaKernelNodeParams kp;
     memset(&kp, 0, sizeof(kp));
     kp.func = (void *)k_set_params;
@@ -777,6 +793,9 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     D.R = cfg->ctx_frames + 2 * cfg->max_spec, D.W = cfg->ctx_frames, D.n_streams = cfg->n_streams;
     D.norm = cfg->norm, D.eps = cfg->norm_eps, D.t_scale = cfg->t_scale;
     D.page_elems = (size_t)D.H * D.T * D.dh;
+    c->lim.n_streams = cfg->n_streams, c->lim.W = cfg->ctx_frames, c->lim.n_slots = NFD_COND_SLOTS;
+    c->lim.n_actions = cfg->n_actions, c->lim.max_frames = NFD_MAX_PASS_FRAMES;
+    c->lim.pend_slots = cfg->n_streams * cfg->max_spec;
     c->n_committed.assign(cfg->n_streams, 0);
     c->n_tentative.assign(cfg->n_streams, 0);
     c->n_pending.assign(cfg->n_streams, 0);
@@ -815,7 +834,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
     A((void **)&c->x0_prev, (size_t)NF * c->frame_elems() * 4);
     A((void **)&c->d_sp, sizeof(StepParams));
     A((void **)&c->d_hash, 8);
-    A((void **)&c->d_status, 4);
+    A((void **)&c->d_status, 16);
     A((void **)&c->d_rope, sizeof(RopeTab));
     A((void **)&c->rope_cs, Mmax * (D.dh / 2) * sizeof(float2));
     if (rc == NFD_OK) {
@@ -843,7 +862,7 @@ int nfd_create(nfd_ctx **out, const nfd_weights *w, const nfd_cfg *cfg, void *cu
         cudaError_t e = cudaMemcpyAsync(c->d_rope, &rt, sizeof(rt), cudaMemcpyHostToDevice, c->st);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->kc, 0, cache_elems * c->esz, c->st);
         if (e == cudaSuccess) e = cudaMemsetAsync(c->vc, 0, cache_elems * c->esz, c->st);
-        if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 4, c->st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 16, c->st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->st);
         if (e != cudaSuccess) {
             fprintf(stderr, "libnfd: create: %s\n", cudaGetErrorString(e));
@@ -957,15 +976,13 @@ int nfd_warm_modulation(nfd_ctx *c) {
         const int nc = c->h_sp.nc;
         if (nc == 0) continue;
         c->cls = CLS_PARAMS;
-        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp);
+        PLAUNCH(c, k_set_params, 1, 256, 0, c->h_sp, c->d_sp, c->lim, c->d_status);
         if (c->bf16_mode)
             enqueue_conditioning<bf16>(c, (int)fr.size());
         else
             enqueue_conditioning<float>(c, (int)fr.size());
-        cudaError_t e = cudaGetLastError();
-        if (e == cudaSuccess) e = c->launch_err;
+        const cudaError_t e = take_launch_err(c);
         if (e != cudaSuccess) {
-            c->launch_err = cudaSuccess;
             for (int r = 0; r < nc; ++r) c->cond_slots[c->h_sp.cd[r].slot] = nfd_ctx::CondSlot();
             fprintf(stderr, "libnfd: %s\n", cudaGetErrorString(e));
             return NFD_E_CUDA;
@@ -1054,7 +1071,10 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
     const int eg = (int)((ne + 255) / 256);
     // Section 4.1 "Sampling": start from pure noise at t' = pi/2
     c->cls = CLS_SAMPLER;
-    PLAUNCH(c, k_axpby, eg, 256, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
+    // (test switch: a block size beyond the device's limit, which the runtime refuses on the host)
+    const int blk0 = c->test_fail_launch ? 4096 : 256;
+    c->test_fail_launch = false;
+    PLAUNCH(c, k_axpby, eg, blk0, 0, c->xp, (float)sd, noise, 0.f, (const float *)nullptr, ne);
     std::vector<float> tv(n);
     for (int s = 0; s < S; ++s) {
         const double tp = 0.5 * M_PI * (double)(S - s) / (double)S;
@@ -1101,8 +1121,7 @@ int nfd_speculate_batched(nfd_ctx *c, int n, const int *streams, int k, const in
         PLAUNCH(c, k_sampler_post, eg, 256, 0, c->xp, (const float *)c->vbuf, z, x0_out, (float)(sd * alpha),
                 (float)(-sd * t), (float)cn, (float)sn_next, ne);
     }
-    CK(cudaGetLastError());
-    CK(c->launch_err);
+    CK(take_launch_err(c));
     if (!c->lazy) {
         std::vector<int> fa((size_t)n * k);
         for (int i = 0; i < n; ++i)
@@ -1163,8 +1182,7 @@ int nfd_sample_dpmpp(nfd_ctx *c, int stream, int k, int action, int n_evals, con
         PLAUNCH(c, k_dpmpp_update, eg, 256, 0, c->xp, (const float *)c->vbuf, c->x0_prev, tf, (float)a, (float)b,
                 (float)cc, i == M ? x0_out : (float *)nullptr, c->cfg.sigma_d, ne);
     }
-    CK(cudaGetLastError());
-    CK(c->launch_err);
+    CK(take_launch_err(c));
     std::vector<int> fa(k, action);
     return commit_pass(c, 1, &stream, k, fa.data(), x0_out, ctx_noise, true);
 }
@@ -1278,13 +1296,48 @@ int nfd_attention(nfd_ctx *c, const void *q, const void *k, const void *v, int n
         p.fr[j].first_new = n_kv - n_q;
     }
     c->cls = CLS_PARAMS;
-    PLAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp);
+    PLAUNCH(c, k_set_params, 1, 256, 0, p, c->d_sp, c->lim, c->d_status);
     if (c->bf16_mode)
         launch_attention<bf16>(c, n_q, 0);
     else
         launch_attention<float>(c, n_q, 0);
-    CK(cudaGetLastError());
+    CK(take_launch_err(c));
     CK(cudaMemcpyAsync(out, c->abuf, qbytes, cudaMemcpyDeviceToDevice, c->st));
+    return NFD_OK;
+}
+
+// Section 4.2: frames i .. i+k-1 were generated under actions[i]; the leading frames whose true action equals
+// it are verified, the first mismatch and everything after it are discarded.  Frame i itself used its true
+// action, so the count is at least 1.
+int nfd_accepted_count(const int *actions, int n, int i, int k) {
+    if (!actions) return NFD_E_NULLPTR;
+    if (n < 1 || i < 0 || i >= n || k < 1) return NFD_E_RANGE;
+    int m = 1;
+    while (m < k && i + m < n && actions[i + m] == actions[i]) ++m;
+    return m;
+}
+
+int nfd_debug_read(nfd_ctx *c, const char *name, float *out, long long n_elems) {
+    if (!c || !name || !out) return NFD_E_NULLPTR;
+    if (!aligned16(out)) return NFD_E_ALIGN;
+    const size_t rows = (size_t)NFD_MAX_PASS_FRAMES * c->D.T;
+    const void *src = nullptr;
+    size_t cap = 0;
+    bool is_f32 = !c->bf16_mode;
+    if (!strcmp(name, "z")) src = c->z, cap = rows * c->D.d, is_f32 = true;
+    else if (!strcmp(name, "hbuf")) src = c->hbuf, cap = rows * c->D.d;
+    else if (!strcmp(name, "qbuf")) src = c->qbuf, cap = rows * c->D.d;
+    else if (!strcmp(name, "abuf")) src = c->abuf, cap = rows * c->D.d;
+    else if (!strcmp(name, "mbuf")) src = c->mbuf, cap = rows * c->D.dm;
+    else return NFD_E_RANGE;
+    if (n_elems < 1 || (size_t)n_elems > cap) return NFD_E_RANGE;
+    c->cls = CLS_CACHE;
+    const int grid = (int)(((size_t)n_elems + 255) / 256);
+    if (is_f32)
+        LAUNCH(c, (k_to_f32<float>), grid, 256, 0, (const float *)src, out, (size_t)n_elems);
+    else
+        LAUNCH(c, (k_to_f32<bf16>), grid, 256, 0, (const bf16 *)src, out, (size_t)n_elems);
+    CK(cudaGetLastError());
     return NFD_OK;
 }
 
@@ -1346,6 +1399,34 @@ int nfd_set_option(nfd_ctx *c, const char *name, int value) {
         for (auto &cs : c->cond_slots) cs = nfd_ctx::CondSlot();
         return NFD_OK;
     }
+    if (!strcmp(name, "l2_prefetch")) {
+        c->l2_prefetch = value != 0;
+        return NFD_OK;
+    }
+    if (!strcmp(name, "kv_prefetch")) {
+        c->kv_prefetch = value != 0;
+        return NFD_OK;
+    }
+    if (!strcmp(name, "clear_status")) {
+        CK(cudaMemsetAsync(c->d_status, 0, 4, c->st));
+        return NFD_OK;
+    }
+    if (!strcmp(name, "test_wait_limit_us") || !strcmp(name, "test_skip_stage")) {
+        // words 1 and 2 of the status block (see nfd_sm100.cuh); 0 restores normal operation
+        if (value < 0) return NFD_E_RANGE;
+        const int word = name[5] == 'w' ? 1 : 2;
+        c->test_words[word] = value;
+        CK(cudaMemcpyAsync(c->d_status + word, &c->test_words[word], 4, cudaMemcpyHostToDevice, c->st));
+        return NFD_OK;
+    }
+    if (!strcmp(name, "test_fail_launch")) {
+        c->test_fail_launch = value != 0;
+        return NFD_OK;
+    }
+    if (!strcmp(name, "test_corrupt_desc")) {
+        c->test_corrupt_desc = value != 0;
+        return NFD_OK;
+    }
     if (!strcmp(name, "lazy_commit")) {
         if (!value)
             for (int s = 0; s < c->cfg.n_streams; ++s) RET(flush_pending(c, s));
@@ -1385,7 +1466,8 @@ int nfd_trace_read(nfd_ctx *c, void *host_buf, int cap) {
 // ---------------------------------------------------------------------------
 #define NFD_NOALLOC_SCRATCH_BYTES 4096
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NFD_NOALLOC_SCRATCH_BYTES];
-static_assert(sizeof(StepParams) <= NFD_NOALLOC_SCRATCH_BYTES, "pass descriptor must fit the static scratch");
+#define NFD_NOALLOC_STATUS_OFFSET 3072       // four status ints behind the descriptor
+static_assert(sizeof(StepParams) <= NFD_NOALLOC_STATUS_OFFSET, "pass descriptor must fit the static scratch");
 
 #define NFD_NOALLOC_MAX_DEVICES 64
 // Device address of g_noalloc_scratch per device ordinal.  In host code the
@@ -1424,6 +1506,11 @@ extern "C" int nfd_attention_noalloc(const void *q, const void *k_pages, const v
         return NFD_E_RANGE;
     }
     if (n_kv_frames < n_q_frames || n_kv_frames > 65536) return NFD_E_RANGE;
+    // sizes whose products the kernel forms in 32-bit integers (model width, rows of the pass, grid)
+    if (n_heads > 1024 || tokens_per_frame > (1 << 20)) return NFD_E_RANGE;
+    const long long rows_ll = (long long)n_q_frames * tokens_per_frame;
+    const long long warps_ll = rows_ll * n_heads;
+    if (rows_ll > 0x7fffffffLL / 4 || (warps_ll + 3) / 4 > 0x7fffffffLL) return NFD_E_RANGE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     int dev = -1;
     CK(cudaGetDevice(&dev));
@@ -1436,6 +1523,8 @@ extern "C" int nfd_attention_noalloc(const void *q, const void *k_pages, const v
         g_noalloc_dev_ptr[dev] = p;
     }
     StepParams *d_sp = (StepParams *)g_noalloc_dev_ptr[dev];
+    // the descriptor check of k_set_params records a failure in a status word; it lives in the same array
+    int *d_stat = (int *)((unsigned char *)g_noalloc_dev_ptr[dev] + NFD_NOALLOC_STATUS_OFFSET);
     Dims D;
     memset(&D, 0, sizeof(D));
     D.L = 1, D.H = n_heads, D.dh = head_dim, D.d = n_heads * head_dim, D.T = tokens_per_frame;
@@ -1451,10 +1540,12 @@ extern "C" int nfd_attention_noalloc(const void *q, const void *k_pages, const v
         p.fr[j].win_first = p.fr[j].frame - window > 0 ? p.fr[j].frame - window : 0;
         p.fr[j].first_new = n_kv_frames - n_q_frames;
     }
+    DescLimits lim;
+    lim.n_streams = 1, lim.W = window, lim.n_slots = 1, lim.n_actions = 1, lim.max_frames = NFD_MAX_PASS_FRAMES;
+    lim.pend_slots = 1;
     // the descriptor is rewritten in full on every call; nothing of the previous call survives
-    k_set_params<<<1, 256, 0, st>>>(p, d_sp);
+    k_set_params<<<1, 256, 0, st>>>(p, d_sp, lim, d_stat);
     CK(cudaGetLastError());
     if (dtype == NFD_DTYPE_BF16) return noalloc_launch<bf16>(st, d_sp, D, n_q_frames, q, k_pages, v_pages, out);
     return noalloc_launch<float>(st, d_sp, D, n_q_frames, q, k_pages, v_pages, out);
 }
-

@@ -20,9 +20,10 @@
 // (max, sum, O) state, S accumulator and P tile, so that one group's
 // exponentials overlap the other's tensor-memory traffic and UMMAs.
 // At the end the two groups' states are merged in shared memory.  A key range
-// longer than CH blocks is split over several CTAs; each writes its unnormalised
-// (O, m, l) state, and the CTA that finishes last (a counter per query tile)
-// merges the states in split order and writes the output.
+// longer than CH blocks is split over several CTAs; each leaves its unnormalised
+// (O, m, l) state in a tile of shared memory and publishes it with one bulk copy;
+// the CTA that finishes last (a counter per query tile) pulls the other tiles in
+// with bulk copies, merges the states in split order and writes the output.
 // CH depends only on the configuration, so a frame's result does not depend on
 // which other frames share its pass.
 #pragma once
@@ -36,22 +37,22 @@ struct AttnPlan {
     int MAXSPLIT = 0;    // splits of the longest window
 };
 
-#ifndef ATTN_POLY_PAIR
-#define ATTN_POLY_PAIR (-1)     // which of the 4 column pairs of an 8-column group uses ex2_poly (-1: none)
-#endif
-
 template <int KB> struct AttnCfg {
     static constexpr int NST = 4;                          // K/V ring stages
     static constexpr int Q_BYTES = 128 * 128;
     static constexpr int P_BYTES = 2 * 128 * 128;          // one group's P tile: two 64-key atoms
     static constexpr int KV_BYTES = KB * 128;              // one K (or V) block
     static constexpr int RING_BYTES = NST * 2 * KV_BYTES;
-    static constexpr int OROW = 68;                        // floats per parked O row (64 + pad)
-    static constexpr int PARK_BYTES = 128 * OROW * 4 + 128 * 8;           // group 1's state: O rows, then (m, l)
+    // A parked state: 128 rows of 64 floats (256 bytes per row; the 16-byte words of row r are stored at
+    // word index c ^ (r & 15), so that one thread per row writes without bank conflicts), then 128 x (m, l).
+    static constexpr int PARK_O_BYTES = 128 * 256;
+    static constexpr int PARK_BYTES = PARK_O_BYTES + 128 * 8;
+    static constexpr int N_IN = RING_BYTES / PARK_BYTES;   // other splits' states that the K/V ring holds at once
     static constexpr int SMEM = Q_BYTES + 2 * P_BYTES + RING_BYTES + 1024 + 256;
     static constexpr int TMEM_COLS = 512;                  // S0 @0, S1 @128, O0 @256, O1 @320
     static constexpr int THREADS = 320;
-    static_assert(PARK_BYTES <= 2 * P_BYTES, "group 1's parked state must fit the P tiles");
+    static_assert(PARK_BYTES <= 2 * P_BYTES, "the parked state must fit the P tiles");
+    static_assert(N_IN >= 1, "the K/V ring must hold one incoming state");
 };
 
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_bmn(int M, int N) {
@@ -64,20 +65,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// 2^y on the FMA and integer pipes, for a share of the softmax's exponentials: the special-function unit
-// (16 ex2 per clock and SM) is what bounds the softmax at head dimension 64.  Round-to-nearest split
-// y = n + f by the magic-number addition, a cubic for 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below
-// the bf16 rounding of P), n added to the exponent field.  y <= 127; results below 2^-125 are clamped there.
-__device__ __forceinline__ float ex2_poly(float y) {
-    y = fmaxf(y, -125.0f);
-    const float t = y + 12582912.0f;               // 1.5 * 2^23: round(y) lands in the low mantissa bits
-    const float f = y - (t - 12582912.0f);
-    float p = fmaf(0.05517220f, f, 0.24261118f);
-    p = fmaf(p, f, 0.69326091f);
-    p = fmaf(p, f, 0.99992806f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-
 __device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }
@@ -86,31 +73,28 @@ template <int KB>
 __global__ void __launch_bounds__(AttnCfg<KB>::THREADS, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
           const __grid_constant__ CUtensorMap tmV, const StepParams *sp, Dims D, int layer, AttnPlan pl, bf16 *out,
-          float *part_o, float2 *part_ml, unsigned int *counters, int *status) {
+          float *part_o, unsigned int *counters, int *status) {
     using A = AttnCfg<KB>;
     extern __shared__ uint8_t smem_raw[];
     NFD_TRACE_T0();
     const int z = blockIdx.z, j = z / D.H, h = z % D.H;
     const int qt = blockIdx.y, split = blockIdx.x;
-    // the pass descriptor was written by the first kernel of the pass, which completed long ago
+    // the pass descriptor was written by the first kernel of the pass, which completed long ago; the loads
+    // are issued here and first used after the set-up below, which hides their latency
     const FrameDesc fr = sp->fr[j];
-    const int nbt = (fr.frame - fr.win_first + 1) * pl.BPF;      // key blocks of this frame's window
-    const int nsplit = (nbt + pl.CH - 1) / pl.CH;
-    if (split >= nsplit) return;                                  // uniform for the CTA, before any barrier or allocation
-    const int b0 = split * pl.CH;
-    const int nb = min(nbt, b0 + pl.CH) - b0;                     // >= 1
-    const int Nq = sp->nf * D.T;
+    const int nf_pass = sp->nf;
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = smem, *sP = smem + A::Q_BYTES, *sKV = sP + 2 * A::P_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + A::RING_BYTES);
     const uint32_t q_full = smem_u32(bars), kv_full = smem_u32(bars + 1), kv_empty = smem_u32(bars + 1 + A::NST),
-                   s_full = smem_u32(bars + 1 + 2 * A::NST), p_full = s_full + 16, pv_done = s_full + 32;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 1 + 2 * A::NST + 6);
+                   s_full = smem_u32(bars + 1 + 2 * A::NST), p_full = s_full + 16, pv_done = s_full + 32,
+                   in_full = s_full + 48, stagger = s_full + 56;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 1 + 2 * A::NST + 8);
     int *last_flag = reinterpret_cast<int *>(tmem_slot + 1);
-    // group 1 parks its state here after the main loop (the P tiles are free by then)
-    float *parkO = reinterpret_cast<float *>(sP);
-    float2 *parkML = reinterpret_cast<float2 *>(sP + 128 * A::OROW * 4);
+    // states are parked here after the main loop (the P tiles are free by then)
+    uint8_t *parkO = sP;
+    float2 *parkML = reinterpret_cast<float2 *>(sP + A::PARK_O_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (warp == 0 && lane == 0) {
@@ -127,6 +111,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             mbar_init(p_full + 8 * g, 128);
             mbar_init(pv_done + 8 * g, 1);
         }
+        mbar_init(in_full, 1);
+        mbar_init(stagger, 128);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -138,7 +124,18 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 0) {
+    const int nbt = (fr.frame - fr.win_first + 1) * pl.BPF;      // key blocks of this frame's window
+    const int nsplit = (nbt + pl.CH - 1) / pl.CH;
+    // a CTA beyond the splits of its frame's window has nothing to do (uniform for the CTA): it skips the
+    // roles below and leaves by the common exit
+    const bool idle = split >= nsplit;
+    const int b0 = split * pl.CH;
+    const int nb = idle ? 0 : min(nbt, b0 + pl.CH) - b0;          // >= 1 unless idle
+    const int Nq = nf_pass * D.T;
+
+    if (idle) {
+        // nothing
+    } else if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const int page_rows = D.H * D.T;
@@ -150,6 +147,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 // pages of frames written earlier than this pass may be fetched before the predecessor finishes
                 if (!waited && (g >= fr.first_new || b >= A::NST)) {
                     pdl_wait();
+                    NFD_TRACE_MARK(TRK_OTHER + 10);
                     waited = true;
                     mbar_expect_tx(q_full, A::Q_BYTES);
                     tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
@@ -184,8 +182,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 umma_commit(s_full + 8 * g);
                 return true;
             };
+            // The two groups share each scheduler's special-function unit.  Started together they stay in step:
+            // both wait for their S at the same time and both exponentiate at the same time, at half the
+            // rate each.  Group 1's first S is therefore issued only when group 0 is half way through its
+            // first block, which puts the groups in opposite phases: one exponentiates while the other waits.
             if (ok) ok = issue_s(0);
-            if (ok && nb > 1) ok = issue_s(1);
+            if (ok && nb > 1) ok = mbar_wait(stagger, 0, status) && issue_s(1);
             for (int b = 0; b < nb && ok; ++b) {
                 const int g = b & 1, s = b % A::NST;
                 ok = mbar_wait(p_full + 8 * g, (b >> 1) & 1, status);
@@ -223,6 +225,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             ok = mbar_wait(s_full + 8 * g, i & 1, status);
             if (!ok) break;
             tc_fence_after();
+            if (i == 0) NFD_TRACE_MARK_T(TRK_OTHER + 11, 64);
             // pass 1 over S: row maximum (all loads in flight together; the values die right after)
             float mx;
             {
@@ -277,17 +280,16 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 uint32_t *cur = ((cc >> 4) & 1) ? sb : sa, *nxt = ((cc >> 4) & 1) ? sa : sb;
                 tmem_ld_wait();
                 if (cc + 16 < KB) tmem_ld16(tS + cc + 16, nxt);
+                if (cc == (KB / 32) * 16 && g == 0 && i == 0) mbar_arrive(stagger);     // see the UMMA issuer
 #pragma unroll
                 for (int u2 = 0; u2 < 2; ++u2) {
                     uint32_t pk[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        // one pair in four goes to the FMA pipes (ex2_poly)
                         const float2 y = ffma2(make_float2(__uint_as_float(cur[8 * u2 + 2 * u]),
                                                            __uint_as_float(cur[8 * u2 + 2 * u + 1])),
                                                make_float2(c, c), make_float2(-m_run, -m_run));
-                        const float p0 = (u == ATTN_POLY_PAIR) ? ex2_poly(y.x) : ex2_approx(y.x);
-                        const float p1 = (u == ATTN_POLY_PAIR) ? ex2_poly(y.y) : ex2_approx(y.y);
+                        const float p0 = ex2_approx(y.x), p1 = ex2_approx(y.y);
                         ls2[u] = fadd2(ls2[u], make_float2(p0, p1));
                         const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
                         pk[u] = *reinterpret_cast<const uint32_t *>(&hp);
@@ -302,6 +304,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             tc_fence_before();
             mbar_arrive(p_full + 8 * g);
         }
+        NFD_TRACE_MARK_T(TRK_OTHER + 12, 64);
         // this group's O accumulator (unnormalised, relative to m_run)
         float O[64];
 #pragma unroll
@@ -327,12 +330,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         }
         const int row = qt * 128 + trow;
         const size_t item_q = (size_t)z * pl.QT + qt;      // (frame, head, query tile)
+        // 16-byte word c of row r of a parked state
+        auto park_word = [](uint8_t *base, int r, int c) { return reinterpret_cast<float4 *>(base + r * 256 + ((c ^ (r & 15)) << 4)); };
         // ---- the two groups of this CTA first: group 1 parks its state, group 0 folds it in ----
-        named_bar_sync(1, 256);                            // both groups are past their last UMMA: the P tiles are free
+        named_bar_sync(1, 256);                            // both groups are past their last UMMA: P tiles and ring are free
         if (g == 1) {
-            float4 *po = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);
 #pragma unroll
-            for (int e = 0; e < 64; e += 4) po[e >> 2] = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
+            for (int e = 0; e < 64; e += 4) *park_word(parkO, trow, e >> 2) = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
             parkML[trow] = make_float2(m_run, l_run);
         }
         named_bar_sync(1, 256);
@@ -342,14 +346,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             m_cta = fmaxf(m_run, ml1.x);
             const float w0 = ex2_approx(m_run - m_cta), w1 = ex2_approx(ml1.x - m_cta);
             l_cta = l_run * w0 + ml1.y * w1;
-            const float4 *po = reinterpret_cast<const float4 *>(parkO + (size_t)trow * A::OROW);
 #pragma unroll
             for (int e = 0; e < 64; e += 4) {
-                const float4 v = po[e >> 2];
+                const float4 v = *park_word(parkO, trow, e >> 2);
                 O[e] = fmaf(O[e], w0, v.x * w1), O[e + 1] = fmaf(O[e + 1], w0, v.y * w1);
                 O[e + 2] = fmaf(O[e + 2], w0, v.z * w1), O[e + 3] = fmaf(O[e + 3], w0, v.w * w1);
             }
         }
+        NFD_TRACE_MARK_T(TRK_OTHER + 13, 64);
         if (nsplit == 1) {
             if (g == 0 && row < D.T) {
                 const float inv = 1.0f / l_cta;
@@ -364,107 +368,104 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             }
         } else {
             // ---- publish this CTA's state; the CTA that finishes last merges the splits in split order ----
-            const size_t st0 = item_q * pl.MAXSPLIT * 128;                           // first state row of this query tile
+            // state tiles in global memory: [query tile][split] x PARK_BYTES, laid out like the parked tile
+            uint8_t *gstates = reinterpret_cast<uint8_t *>(part_o);
+            const size_t st0 = item_q * pl.MAXSPLIT;
             if (g == 0) {
-                const size_t item = st0 + (size_t)split * 128 + trow;
-                float4 *po4 = reinterpret_cast<float4 *>(part_o + item * 64);
-                float4 *ps4 = reinterpret_cast<float4 *>(parkO + (size_t)trow * A::OROW);     // own copy for the merge
+                // (each thread rewrites only the row it has just read)
 #pragma unroll
-                for (int e = 0; e < 64; e += 4) {
-                    const float4 v = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
-                    po4[e >> 2] = v;
-                    ps4[e >> 2] = v;
-                }
-                part_ml[item] = make_float2(m_cta, l_cta);
+                for (int e = 0; e < 64; e += 4) *park_word(parkO, trow, e >> 2) = make_float4(O[e], O[e + 1], O[e + 2], O[e + 3]);
                 parkML[trow] = make_float2(m_cta, l_cta);
-                __threadfence();
+                fence_proxy_async_smem();                  // the bulk copy below reads what this thread wrote
             }
             named_bar_sync(1, 256);
             if (threadIdx.x == 64) {
+                bulk_store_s2g(gstates + (st0 + split) * A::PARK_BYTES, smem_u32(parkO), A::PARK_BYTES);
+                bulk_commit();
+                bulk_wait_all();                           // the tile has been written
+                __threadfence();
                 const unsigned int prev = atomicAdd(counters + item_q, 1u);
                 const int last = prev == (unsigned int)(nsplit - 1);
-                if (last) counters[item_q] = 0;            // ready for the next launch
+                if (last) {
+                    counters[item_q] = 0;                  // ready for the next launch
+                    __threadfence();
+                }
                 *last_flag = last;
             }
+            NFD_TRACE_MARK_T(TRK_OTHER + 14, 64);
             named_bar_sync(1, 256);
             if (*last_flag) {
-                __threadfence();
-                // an item = 8 adjacent output columns of a row; two items per thread and round, so that the
-                // loads of both (all splits, four at a time) are in flight together
-                for (int it0 = (int)threadIdx.x - 64; it0 < 128 * 8; it0 += 512) {
-                    int r[2], ch[2];
-                    bool live[2];
-                    float acc[2][8], l[2], mx[2];
+                // an item = 8 adjacent output columns of a row; four items per thread (256 threads, 128 x 8 items).
+                // The other splits' states come in through the K/V ring, N_IN at a time; every item keeps a
+                // running (max, sum, accumulator) and takes the splits in split order whatever N_IN is.
+                const int et = (int)threadIdx.x - 64;
+                float acc[4][8], l[4], mx[4];
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        const int it = it0 + q * 256;
-                        r[q] = it >> 3, ch[q] = it & 7;
-                        live[q] = it < 128 * 8 && qt * 128 + r[q] < D.T;
-                        l[q] = 0.f, mx[q] = -INFINITY;
+                for (int q = 0; q < 4; ++q) {
+                    l[q] = 0.f, mx[q] = -INFINITY;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[q][e] = 0.f;
+                    for (int e = 0; e < 8; ++e) acc[q][e] = 0.f;
+                }
+                uint32_t in_phase = 0;
+                bool ok_in = true;
+                for (int s0 = 0, s1 = 0; s0 < nsplit && ok_in; s0 = s1) {
+                    // this round: splits s0 .. s1-1; the own split (if in range) is read from the parked tile
+                    int n_in = 0;
+                    while (s1 < nsplit && (n_in < A::N_IN || s1 == split)) n_in += (s1 != split), ++s1;
+                    if (s0 > 0) named_bar_sync(1, 256);    // everyone is done reading the ring's previous contents
+                    if (threadIdx.x == 64 && n_in > 0) {
+                        fence_proxy_async_all();
+                        mbar_expect_tx(in_full, (uint32_t)n_in * A::PARK_BYTES);
+                        int slot = 0;
+                        for (int sidx = s0; sidx < s1; ++sidx)
+                            if (sidx != split)
+                                bulk_load_g2s(smem_u32(sKV + (slot++) * A::PARK_BYTES), gstates + (st0 + sidx) * A::PARK_BYTES,
+                                              A::PARK_BYTES, in_full);
                     }
-                    for (int s0 = 0; s0 < nsplit; s0 += 4) {
-                        // this CTA's own state comes from shared memory (same values as its published copy)
-                        float2 ml[2][4];
-                        float4 v0[2][4], v1[2][4];
+                    if (n_in > 0) {
+                        ok_in = mbar_wait(in_full, in_phase, status);
+                        in_phase ^= 1;
+                        if (!ok_in) break;
+                    }
+                    int slot = 0;
+                    for (int sidx = s0; sidx < s1; ++sidx) {
+                        uint8_t *base = sidx == split ? parkO : sKV + (slot++) * A::PARK_BYTES;
+                        const float2 *bml = reinterpret_cast<const float2 *>(base + A::PARK_O_BYTES);
 #pragma unroll
-                        for (int q = 0; q < 2; ++q) {
-                            if (!live[q]) continue;
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const int sidx = s0 + u < nsplit ? s0 + u : nsplit - 1;
-                                if (sidx == split) {
-                                    ml[q][u] = parkML[r[q]];
-                                    const float4 *po =
-                                        reinterpret_cast<const float4 *>(parkO + (size_t)r[q] * A::OROW + ch[q] * 8);
-                                    v0[q][u] = po[0], v1[q][u] = po[1];
-                                } else {
-                                    const size_t item = st0 + (size_t)sidx * 128 + r[q];
-                                    ml[q][u] = __ldcg(&part_ml[item]);
-                                    const float4 *po = reinterpret_cast<const float4 *>(part_o + item * 64 + ch[q] * 8);
-                                    v0[q][u] = __ldcg(po), v1[q][u] = __ldcg(po + 1);
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int q = 0; q < 2; ++q) {
-                            if (!live[q]) continue;
-                            float mb = mx[q];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u)
-                                if (s0 + u < nsplit) mb = fmaxf(mb, ml[q][u].x);
-                            const float fo = ex2_approx(mx[q] - mb);   // rescale of what was merged so far (0 at first)
-                            l[q] *= fo;
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) acc[q][e] *= fo;
+                        for (int q = 0; q < 4; ++q) {
+                            const int it = et + q * 256, r = it >> 3, ch = it & 7;
+                            const float2 ml = bml[r];
+                            const float4 v0 = *park_word(base, r, 2 * ch), v1 = *park_word(base, r, 2 * ch + 1);
+                            const float mb = fmaxf(mx[q], ml.x);
+                            // (a state without any key has m = -inf, l = 0: it must count for nothing)
+                            const float fo = mx[q] == mb ? 1.0f : ex2_approx(mx[q] - mb);
+                            const float w = ml.x == -INFINITY ? 0.f : ex2_approx(ml.x - mb);
                             mx[q] = mb;
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                if (s0 + u < nsplit) {
-                                    const float w = ex2_approx(ml[q][u].x - mb);
-                                    l[q] = fmaf(ml[q][u].y, w, l[q]);
-                                    acc[q][0] = fmaf(v0[q][u].x, w, acc[q][0]), acc[q][1] = fmaf(v0[q][u].y, w, acc[q][1]);
-                                    acc[q][2] = fmaf(v0[q][u].z, w, acc[q][2]), acc[q][3] = fmaf(v0[q][u].w, w, acc[q][3]);
-                                    acc[q][4] = fmaf(v1[q][u].x, w, acc[q][4]), acc[q][5] = fmaf(v1[q][u].y, w, acc[q][5]);
-                                    acc[q][6] = fmaf(v1[q][u].z, w, acc[q][6]), acc[q][7] = fmaf(v1[q][u].w, w, acc[q][7]);
-                                }
-                            }
+                            l[q] = fmaf(ml.y, w, l[q] * fo);
+                            acc[q][0] = fmaf(v0.x, w, acc[q][0] * fo), acc[q][1] = fmaf(v0.y, w, acc[q][1] * fo);
+                            acc[q][2] = fmaf(v0.z, w, acc[q][2] * fo), acc[q][3] = fmaf(v0.w, w, acc[q][3] * fo);
+                            acc[q][4] = fmaf(v1.x, w, acc[q][4] * fo), acc[q][5] = fmaf(v1.y, w, acc[q][5] * fo);
+                            acc[q][6] = fmaf(v1.z, w, acc[q][6] * fo), acc[q][7] = fmaf(v1.w, w, acc[q][7] * fo);
                         }
                     }
+                }
+                if (ok_in) {
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        if (!live[q]) continue;
-                        const float inv = 1.0f / l[q];
+                    for (int q = 0; q < 4; ++q) {
+                        const int it = et + q * 256, r = it >> 3, ch = it & 7;
+                        if (qt * 128 + r < D.T) {
+                            const float inv = 1.0f / l[q];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) acc[q][u] *= inv;
-                        *reinterpret_cast<uint4 *>(out + (size_t)(j * D.T + qt * 128 + r[q]) * D.d + h * 64 + ch[q] * 8) =
-                            pack_bf16x8(acc[q]);
+                            for (int u = 0; u < 8; ++u) acc[q][u] *= inv;
+                            *reinterpret_cast<uint4 *>(out + (size_t)(j * D.T + qt * 128 + r) * D.d + h * 64 + ch * 8) =
+                                pack_bf16x8(acc[q]);
+                        }
                     }
                 }
             }
         }
     }
+    NFD_TRACE_MARK_T(TRK_OTHER + 16, 64);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, A::TMEM_COLS);

@@ -24,8 +24,7 @@ struct FastState {
     int n_sm = 148;
     size_t a_rows = 0;     // rows of every activation buffer (NFD_MAX_PASS_FRAMES * T)
     AttnPlan plan;         // KB == 0: tensor-core attention not available for this shape
-    float *part_o = nullptr;           // per-split states of the attention kernel
-    float2 *part_ml = nullptr;
+    float *part_o = nullptr;           // per-split states of the attention kernel: [query tile][split] x PARK_BYTES
     unsigned int *attn_counters = nullptr;   // one per (frame, head, query tile); zero between launches
     size_t cache_rows = 0;
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;   // (ptr, rows, cols, box_rows)
@@ -43,9 +42,10 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
         qres != cudaDriverEntryPointSuccess) {
+        // no silent change of path: without tensor maps a bf16 context would run the plain validation kernels
         cudaGetLastError();
-        fprintf(stderr, "libnfd: cuTensorMapEncodeTiled is unavailable; tensor-core path disabled\n");
-        return NFD_OK;
+        fprintf(stderr, "libnfd: the driver does not provide cuTensorMapEncodeTiled; a bf16 context needs it\n");
+        return NFD_E_CUDA;
     }
     fs.encode = (PFN_encodeTiled)fn;
     int dev = 0;
@@ -70,9 +70,7 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
         pl.MAXSPLIT = ((D.W + 1) * pl.BPF + pl.CH - 1) / pl.CH;
         if (pl.MAXSPLIT > 1) {
             const size_t tiles = (size_t)NFD_MAX_PASS_FRAMES * D.H * pl.QT;
-            const size_t items = tiles * pl.MAXSPLIT * 128;          // one state per split
-            if (cudaMalloc((void **)&fs.part_o, items * 64 * sizeof(float)) != cudaSuccess ||
-                cudaMalloc((void **)&fs.part_ml, items * sizeof(float2)) != cudaSuccess ||
+            if (cudaMalloc((void **)&fs.part_o, tiles * pl.MAXSPLIT * (size_t)AttnCfg<64>::PARK_BYTES) != cudaSuccess ||
                 cudaMalloc((void **)&fs.attn_counters, tiles * sizeof(unsigned int)) != cudaSuccess ||
                 cudaMemset(fs.attn_counters, 0, tiles * sizeof(unsigned int)) != cudaSuccess) {
                 cudaGetLastError();
@@ -87,9 +85,8 @@ static int fast_create(FastState &fs, const Dims &D, bool bf16_mode, cudaStream_
 static void fast_destroy(FastState &fs) {
     fs.maps.clear();
     if (fs.part_o) cudaFree(fs.part_o);
-    if (fs.part_ml) cudaFree(fs.part_ml);
     if (fs.attn_counters) cudaFree(fs.attn_counters);
-    fs.part_o = nullptr, fs.part_ml = nullptr, fs.attn_counters = nullptr;
+    fs.part_o = nullptr, fs.attn_counters = nullptr;
     fs.ready = false;
 }
 
@@ -126,12 +123,9 @@ static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
     cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
     cudaLaunchAttribute attr[2];
     int na = 0;
-    static const bool no_pdl = getenv("NFD_NO_PDL") != nullptr;      // debugging aid: plain stream order
-    if (!no_pdl) {
-        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[na].val.programmaticStreamSerializationAllowed = 1;
-        ++na;
-    }
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
     if (cluster_x > 1) {
         attr[na].id = cudaLaunchAttributeClusterDimension;
         attr[na].val.clusterDim.x = (unsigned)cluster_x, attr[na].val.clusterDim.y = 1, attr[na].val.clusterDim.z = 1;
@@ -177,15 +171,6 @@ template <typename Kern> static void query_gemm_slots(FastState &fs, Kern kern, 
 }
 
 static GemmPlan plan_gemm(const FastState &fs, int M, int N, int K, int tc_kind) {
-    // optional override for tuning: NFD_GEMM_PLAN="kind:BN:S,kind:BN:S,..." (kind = TC_* value, +10 for K > 2048)
-    if (const char *e = getenv("NFD_GEMM_PLAN")) {
-        for (const char *p = e; p && *p;) {
-            int k = 0, bn = 0, s = 0;
-            if (sscanf(p, "%d:%d:%d", &k, &bn, &s) == 3 && k == tc_kind + (K > 2048 ? 10 : 0)) return {bn, s};
-            p = strchr(p, ',');
-            if (p) ++p;
-        }
-    }
     if (fs.force_BN) return {fs.force_BN, fs.force_S};
     const int kind_key = tc_kind + (K > 2048 ? 10 : 0);
     {
@@ -320,7 +305,7 @@ static int launch_attn_tc(FastState &fs, cudaStream_t st, const StepParams *sp, 
     const AttnPlan &pl = fs.plan;
     dim3 grid(pl.MAXSPLIT, pl.QT, nf * D.H);
     cudaError_t e = launch_pdl(kern, grid, dim3(A::THREADS), (size_t)A::SMEM, st, 1, *mq, *mk, *mv, sp, D, layer, pl, out,
-                               fs.part_o, fs.part_ml, fs.attn_counters, fs.d_status);
+                               fs.part_o, fs.attn_counters, fs.d_status);
     if (e != cudaSuccess) {
         fprintf(stderr, "libnfd: tensor-core attention launch failed: %s\n", cudaGetErrorString(e));
         cudaGetLastError();

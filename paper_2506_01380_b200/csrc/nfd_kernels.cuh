@@ -8,15 +8,62 @@
 // ---------------------------------------------------------------------------
 // Pass parameters: first kernel of every pass.
 // ---------------------------------------------------------------------------
+// Every index that the kernels of a pass derive from the descriptor (cache page,
+// modulation row, input and output frame slots) is checked here, once, against
+// the limits of the context before the descriptor reaches device memory.  A
+// frame that fails is recorded (NFD_E_DEVICE in the status latch) and replaced
+// by a harmless one -- batch slot 0, frame j of the pass, seeing only itself, no
+// output -- so that nothing downstream leaves its buffers; the caller learns of
+// it from nfd_status and must treat the cache as lost.
+struct DescLimits {
+    int n_streams, W, n_slots, n_actions, max_frames, pend_slots;
+};
 // It does not release its dependents early: a kernel that starts after this one
 // may read the descriptor before its own wait on the predecessor grid.
-__global__ void k_set_params(StepParams p, StepParams *dst) {
+__global__ void k_set_params(StepParams p, StepParams *dst, DescLimits lim, int *status) {
     NFD_TRACE_T0();
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    const int t = threadIdx.x;
+    bool bad = false;
+    if (t == 0) bad = p.nf < 0 || p.nf > lim.max_frames || p.nc < 0 || p.nc > lim.max_frames;
+    if (t < NFD_MAX_PASS_FRAMES && t < p.nf) {
+        const FrameDesc &f = p.fr[t];
+        bad = bad || f.stream < 0 || f.stream >= lim.n_streams || f.frame < 0 || f.win_first < 0 ||
+              f.win_first > f.frame || f.frame - f.win_first > lim.W || f.first_new < 0 || f.first_new > f.frame ||
+              f.cond_row < 0 || f.cond_row >= lim.n_slots || f.src < 0 || f.src > 1 || f.src_index < 0 ||
+              f.src_index >= (f.src ? lim.pend_slots : lim.max_frames) || f.out_index < -1 ||
+              f.out_index >= lim.max_frames;
+    }
+    if (t >= 64 && t - 64 < NFD_MAX_PASS_FRAMES && t - 64 < p.nc) {
+        const CondDesc &cd = p.cd[t - 64];
+        bad = bad || cd.slot < 0 || cd.slot >= lim.n_slots || cd.action < 0 || cd.action >= lim.n_actions;
+    }
+    if (bad) s_bad = 1;
+    __syncthreads();
+    const bool any_bad = s_bad != 0;
     pdl_wait();
     const int n_words = sizeof(StepParams) / 4;
     const int *src = reinterpret_cast<const int *>(&p);
     int *d = reinterpret_cast<int *>(dst);
     for (int i = threadIdx.x; i < n_words; i += blockDim.x) d[i] = src[i];
+    if (any_bad) {
+        __syncthreads();
+        if (t == 0) {
+            atomicCAS(status, 0, NFD_E_DEVICE);
+            int nf = p.nf;
+            nf = nf < 0 ? 0 : (nf > lim.max_frames ? lim.max_frames : nf);
+            dst->nf = nf;
+            dst->nc = 0;
+        }
+        if (t < NFD_MAX_PASS_FRAMES) {
+            FrameDesc f;
+            f.stream = 0, f.frame = t, f.win_first = t, f.cond_row = 0, f.first_new = 0;
+            f.src = 0, f.src_index = 0, f.out_index = -1;
+            dst->fr[t] = f;
+        }
+    }
     NFD_TRACE_END(TRK_PARAMS);
 }
 
@@ -473,10 +520,11 @@ template <typename TS> struct EpiQKV {
     const float2 *rope_cs;      // [nf*T][dh/2] (cos, sin), used by the tensor-core path
     int n_rows;                 // nf*T: rows of the pass (q is [H][n_rows][dh])
     LnFold ln;                  // folded adaLN in front of this projection (tensor-core path only)
+    int kv_prefetch = 1;        // 0: leave the cached pages alone (option "l2_prefetch")
     // Pull the cached K/V pages that the attention kernel of this layer is about to read towards L2 (the
     // pages of frames before this pass are final); each CTA of the launch takes a slice of every page.
     __device__ __forceinline__ void prefetch(unsigned int cta, unsigned int n_cta) const {
-        if (sizeof(TS) != 2) return;
+        if (sizeof(TS) != 2 || !kv_prefetch) return;
         const FrameDesc fr = sp->fr[0];
         const size_t page_bytes = D.page_elems * sizeof(TS);
         const size_t per = ((page_bytes / n_cta + 15) / 16) * 16;
@@ -905,6 +953,11 @@ __global__ void k_kv_read(Dims D, const TS *cache, int stream, int layer, int fr
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= D.page_elems) return;
     out[i] = to_f(cache[kv_page_offset(D, stream, layer, frame) + i]);
+}
+
+template <typename TS> __global__ void k_to_f32(const TS *src, float *out, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = to_f(src[i]);
 }
 
 // copy [H][n_frames*T][dh] (storage type) into pages of (stream 0, layer) frames 0..n_frames-1

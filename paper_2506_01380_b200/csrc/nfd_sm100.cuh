@@ -3,6 +3,13 @@
 // descriptor construction.  Every wait is bounded: on expiry it records
 // NFD_E_TIMEOUT in the status word and returns false; callers then skip their
 // remaining work and fall through to the common exit path.
+//
+// The status block that every kernel gets is four ints: [0] the latch (0 or the
+// first NFD_E_* recorded), [1] a wait limit in microseconds that replaces the
+// default when it is not 0, [2] a test switch: when it is not 0 the GEMM's TMA
+// producer leaves out its last ring stage, so that the consumer's wait for it
+// runs out (used to show that an expired wait surfaces through nfd_status and
+// leaves the context usable), [3] unused.
 #pragma once
 #include <cuda.h>
 #include "nfd_common.cuh"
@@ -46,9 +53,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *status) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
+    unsigned long long limit = NFD_WAIT_LIMIT_NS;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > NFD_WAIT_LIMIT_NS) {
+        if ((++spins & 0x3ff) == 0) {
+            if (spins == 0x400) {
+                const int us = *reinterpret_cast<volatile int *>(status + 1);
+                if (us > 0) limit = (unsigned long long)us * 1000ull;
+            }
+            if (global_timer_ns() - t0 <= limit) continue;
             atomicCAS(status, 0, NFD_E_TIMEOUT);
             return false;
         }
@@ -99,6 +112,22 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
         "[%2];" ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
 }
+
+// ---- untiled bulk copies (16-byte aligned addresses, sizes a multiple of 16) -----
+__device__ __forceinline__ void bulk_store_s2g(void *gdst, uint32_t ssrc, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all bulk groups of this thread are complete (their writes performed)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_load_g2s(uint32_t sdst, const void *gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sdst),
+                 "l"(gsrc), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// orders generic-proxy accesses before later async-proxy (bulk copy) accesses, all state spaces
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // ---- tcgen05 ----------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {

@@ -45,7 +45,7 @@ EXPORTS = ["nfd_create", "nfd_destroy", "nfd_reset", "nfd_denoise_step", "nfd_de
            "nfd_launch_count", "nfd_set_option", "nfd_warm_modulation", "nfd_strerror", "nfd_profile_begin",
            "nfd_profile_end",
            "nfd_profile_class_count", "nfd_profile_class_name", "nfd_attention_noalloc", "nfd_cond_cache_stats",
-           "nfd_sample_dpmpp"]
+           "nfd_sample_dpmpp", "nfd_accepted_count", "nfd_debug_read"]
 
 
 class NfdError(RuntimeError):
@@ -94,6 +94,8 @@ def load():
     lib.nfd_attention_noalloc.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                           vp, vp]
     lib.nfd_cond_cache_stats.argtypes = [vp, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]
+    lib.nfd_accepted_count.argtypes = [ip, C.c_int, C.c_int, C.c_int]
+    lib.nfd_debug_read.argtypes = [vp, C.c_char_p, vp, C.c_longlong]
     lib.nfd_strerror.argtypes = [C.c_int]
     lib.nfd_strerror.restype = C.c_char_p
     _lib = lib
@@ -124,16 +126,12 @@ def _check(code: int, what: str):
 
 
 def accepted_frames(true_actions, i: int, k: int) -> int:
-    """Host-side verification of a speculation (Section 4.2): frames i .. i+k-1
-    were generated under true_actions[i].  Returns how many leading frames were
-    generated under their true action (always >= 1); pass it to rollback()."""
-    first = true_actions[i]
-    n = 1
-    for j in range(i + 1, min(i + k, len(true_actions))):
-        if true_actions[j] != first:
-            break
-        n += 1
-    return n
+    """nfd_accepted_count: how many of the frames i .. i+k-1, generated under
+    true_actions[i], were generated under their own true action; pass it to rollback()."""
+    n = len(true_actions)
+    r = load().nfd_accepted_count(_ints(true_actions), n, int(i), int(k))
+    _check(0 if r > 0 else (r or -4), "nfd_accepted_count")
+    return r
 
 
 def attention_noalloc(q, k_pages, v_pages, n_q_frames: int, window: int, out, stream=None):
@@ -313,6 +311,15 @@ class NFD:
                                       n_q_frames, n_kv_frames, window, C.c_void_p(o.data_ptr())), "nfd_attention")
         self._exit()
         return o
+
+    def debug_read(self, name: str, n_elems: int):
+        """First n_elems elements of an activation buffer of the last pass, as fp32."""
+        out = torch.empty(int(n_elems), device=self.device, dtype=torch.float32)
+        self._enter()
+        _check(self.lib.nfd_debug_read(self._h, name.encode(), C.c_void_p(out.data_ptr()), int(n_elems)),
+               "nfd_debug_read")
+        self._exit()
+        return out
 
     def status(self) -> int:
         return self.lib.nfd_status(self._h)

@@ -56,7 +56,7 @@ def test_strerror_needs_no_gpu():
     assert lib.nfd_strerror(-5) == b"call not allowed in this cache state"
 
 
-def test_host_side_acceptance_rule_matches_oracle():
+def test_acceptance_rule_in_the_library_matches_oracle():
     import itertools
     from oracle.nfd_oracle import accepted_count
     for n in range(1, 7):
@@ -64,3 +64,15 @@ def test_host_side_acceptance_rule_matches_oracle():
             for k in range(1, 5):
                 for i in range(n):
                     assert N.accepted_frames(list(acts), i, k) == accepted_count(list(acts), i, k)
+
+
+def test_accepted_count_argument_checks():
+    from paper_2506_01380_b200 import nfd as N
+    lib = N.load()
+    acts = N._ints([4, 4, 4, 2, 2])
+    assert lib.nfd_accepted_count(acts, 5, 0, 4) == 3
+    assert lib.nfd_accepted_count(acts, 5, 3, 4) == 2
+    assert lib.nfd_accepted_count(acts, 5, 4, 4) == 1
+    assert lib.nfd_accepted_count(acts, 5, 5, 4) == -4
+    assert lib.nfd_accepted_count(None, 5, 0, 4) == -2
+    assert lib.nfd_accepted_count(acts, 5, 0, 0) == -4
