@@ -8,17 +8,31 @@
 //     S  = Q K^T          UMMA 128 x KB x 64, operands in shared memory (TMA),
 //                         accumulator in tensor memory
 //     P  = exp2(S*c - m)  one thread per query row: TMEM -> registers, running
-//                         max / sum, bf16 P written to shared memory
-//     O += P V            UMMA 128 x 64 x KB, V used straight from its page
-//                         (MN-major B operand), accumulated in tensor memory
+//                         max / sum, bf16 P written back to tensor memory over
+//                         the first half of the S columns it came from
+//     O += P V            UMMA 128 x 64 x KB, P read from tensor memory, V used
+//                         straight from its page (MN-major B operand in shared
+//                         memory), accumulated in tensor memory
 // The reference maximum m of a row is raised only when a block's maximum exceeds
 // it by more than 2^8; only then is the row's O accumulator rescaled (in tensor
 // memory), so that in the steady state O is never read back.  The final
 // normalisation by the running sum makes the result independent of that choice.
 // Warp 0 = TMA producer, warp 1 = UMMA issuer, warps 2-5 and 6-9 = two softmax
 // groups.  Group g takes the key blocks b with b % 2 == g and keeps its own
-// (max, sum, O) state, S accumulator and P tile, so that one group's
-// exponentials overlap the other's tensor-memory traffic and UMMAs.
+// (max, sum, O) state and P tile, so that one group's exponentials overlap the
+// other's tensor-memory traffic and UMMAs.  S has three accumulators in tensor
+// memory, block b using number b % 3, and S(b + 3) is issued right behind
+// P V(b), which reads P(b) from that accumulator (the tensor pipe takes its
+// instructions in order): a group finds its next S ready when it comes back for
+// it, instead of waiting for the issue, the product and the completion signal
+// each time.  P never passes through shared memory: the kernel is bound by the
+// rate at which the tensor pipe gets its operands out of shared memory, and a
+// P tile there would be written once and read once more per block.
+// K blocks go through a ring of three stages (stage b % 3; a stage is free again
+// when S(b) is complete, which the barrier of accumulator b % 3 tells), V blocks
+// through a ring of four (free when P V of its block is complete).  Two
+// completion signals per block are all the issuing thread sends, and that
+// thread is the busiest of the kernel.
 // At the end the two groups' states are merged in shared memory.  A key range
 // longer than CH blocks is split over several CTAs; each leaves its unnormalised
 // (O, m, l) state in a tile of shared memory and publishes it with one bulk copy;
@@ -38,18 +52,19 @@ struct AttnPlan {
 };
 
 template <int KB> struct AttnCfg {
-    static constexpr int NST = 4;                          // K/V ring stages
+    static constexpr int NK = 3;                           // K ring stages = S accumulators
+    static constexpr int NV = 4;                           // V ring stages
     static constexpr int Q_BYTES = 128 * 128;
     static constexpr int P_BYTES = 2 * 128 * 128;          // one group's P tile: two 64-key atoms
     static constexpr int KV_BYTES = KB * 128;              // one K (or V) block
-    static constexpr int RING_BYTES = NST * 2 * KV_BYTES;
+    static constexpr int RING_BYTES = (NK + NV) * KV_BYTES;
     // A parked state: 128 rows of 64 floats (256 bytes per row; the 16-byte words of row r are stored at
     // word index c ^ (r & 15), so that one thread per row writes without bank conflicts), then 128 x (m, l).
     static constexpr int PARK_O_BYTES = 128 * 256;
     static constexpr int PARK_BYTES = PARK_O_BYTES + 128 * 8;
     static constexpr int N_IN = RING_BYTES / PARK_BYTES;   // other splits' states that the K/V ring holds at once
     static constexpr int SMEM = Q_BYTES + 2 * P_BYTES + RING_BYTES + 1024 + 256;
-    static constexpr int TMEM_COLS = 512;                  // S0 @0, S1 @128, O0 @256, O1 @320
+    static constexpr int TMEM_COLS = 512;                  // S0 @0, S1 @128, S2 @256, O0 @384, O1 @448
     static constexpr int THREADS = 320;
     static_assert(PARK_BYTES <= 2 * P_BYTES, "the parked state must fit the P tiles");
     static_assert(N_IN >= 1, "the K/V ring must hold one incoming state");
@@ -87,10 +102,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = smem, *sP = smem + A::Q_BYTES, *sKV = sP + 2 * A::P_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(sKV + A::RING_BYTES);
-    const uint32_t q_full = smem_u32(bars), kv_full = smem_u32(bars + 1), kv_empty = smem_u32(bars + 1 + A::NST),
-                   s_full = smem_u32(bars + 1 + 2 * A::NST), p_full = s_full + 16, pv_done = s_full + 32,
-                   in_full = s_full + 48, stagger = s_full + 56;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 1 + 2 * A::NST + 8);
+    // barriers: q_full | k_full[NK] | s_full[NK] | v_full[NV] | v_empty[NV] | p_full[2] | in_full
+    const uint32_t q_full = smem_u32(bars), k_full = q_full + 8, s_full = k_full + 8 * A::NK,
+                   v_full = s_full + 8 * A::NK, v_empty = v_full + 8 * A::NV, p_full = v_empty + 8 * A::NV,
+                   in_full = p_full + 16;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 1 + 2 * A::NK + 2 * A::NV + 3);
     int *last_flag = reinterpret_cast<int *>(tmem_slot + 1);
     // states are parked here after the main loop (the P tiles are free by then)
     uint8_t *parkO = sP;
@@ -102,17 +118,16 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
         mbar_init(q_full, 1);
-        for (int s = 0; s < A::NST; ++s) {
-            mbar_init(kv_full + 8 * s, 1);
-            mbar_init(kv_empty + 8 * s, 1);
+        for (int s = 0; s < A::NK; ++s) {
+            mbar_init(k_full + 8 * s, 1);
+            mbar_init(s_full + 8 * s, 1);
         }
-        for (int g = 0; g < 2; ++g) {
-            mbar_init(s_full + 8 * g, 1);
-            mbar_init(p_full + 8 * g, 128);
-            mbar_init(pv_done + 8 * g, 1);
+        for (int s = 0; s < A::NV; ++s) {
+            mbar_init(v_full + 8 * s, 1);
+            mbar_init(v_empty + 8 * s, 1);
         }
+        for (int g = 0; g < 2; ++g) mbar_init(p_full + 8 * g, 128);
         mbar_init(in_full, 1);
-        mbar_init(stagger, 128);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -139,30 +154,47 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const int page_rows = D.H * D.T;
-            bool waited = false;
-            for (int b = 0; b < nb; ++b) {
-                const int s = b % A::NST;
-                const int blk = b0 + b;
-                const int g = fr.win_first + blk / pl.BPF, kb = blk % pl.BPF;
-                // pages of frames written earlier than this pass may be fetched before the predecessor finishes
-                if (!waited && (g >= fr.first_new || b >= A::NST)) {
-                    pdl_wait();
-                    NFD_TRACE_MARK(TRK_OTHER + 10);
-                    waited = true;
-                    mbar_expect_tx(q_full, A::Q_BYTES);
-                    tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
-                }
-                if (b >= A::NST && !mbar_wait(kv_empty + 8 * s, ((b / A::NST) - 1) & 1, status)) break;
-                const int row = ((fr.stream * D.L + layer) * D.R + (g % D.R)) * page_rows + h * D.T + kb * KB;
-                mbar_expect_tx(kv_full + 8 * s, 2 * A::KV_BYTES);
-                tma_load_2d(smem_u32(sKV + s * 2 * A::KV_BYTES), &tmK, kv_full + 8 * s, 0, row);
-                tma_load_2d(smem_u32(sKV + s * 2 * A::KV_BYTES + A::KV_BYTES), &tmV, kv_full + 8 * s, 0, row);
-            }
-            if (!waited) {
+            uint8_t *sK = sKV, *sV = sKV + A::NK * A::KV_BYTES;
+            bool waited = false, ok = true;
+            auto need_q = [&]() {                // from here on the predecessor's output is needed
+                if (waited) return;
                 pdl_wait();
+                NFD_TRACE_MARK(TRK_OTHER + 10);
+                waited = true;
                 mbar_expect_tx(q_full, A::Q_BYTES);
                 tma_load_2d(smem_u32(sQ), &tmQ, q_full, 0, h * Nq + j * D.T + qt * 128);
+            };
+            auto row_of = [&](int b, bool &is_new) {
+                const int blk = b0 + b;
+                const int g = fr.win_first + blk / pl.BPF, kb = blk % pl.BPF;
+                is_new = g >= fr.first_new;      // pages written by this pass; earlier ones are final already
+                return ((fr.stream * D.L + layer) * D.R + (g % D.R)) * page_rows + h * D.T + kb * KB;
+            };
+            auto load_k = [&](int b) {
+                bool is_new;
+                const int row = row_of(b, is_new), st = b % A::NK;
+                if (is_new || b >= A::NK) need_q();      // a stage is freed by an S product, which needs Q
+                if (b >= A::NK && !mbar_wait(s_full + 8 * st, ((b / A::NK) - 1) & 1, status)) return false;
+                mbar_expect_tx(k_full + 8 * st, A::KV_BYTES);
+                tma_load_2d(smem_u32(sK + st * A::KV_BYTES), &tmK, k_full + 8 * st, 0, row);
+                return true;
+            };
+            auto load_v = [&](int b) {
+                bool is_new;
+                const int row = row_of(b, is_new), st = b % A::NV;
+                if (is_new || b >= A::NV) need_q();
+                if (b >= A::NV && !mbar_wait(v_empty + 8 * st, ((b / A::NV) - 1) & 1, status)) return false;
+                mbar_expect_tx(v_full + 8 * st, A::KV_BYTES);
+                tma_load_2d(smem_u32(sV + st * A::KV_BYTES), &tmV, v_full + 8 * st, 0, row);
+                return true;
+            };
+            // K runs ahead of V: K(b) is used three blocks before V(b)
+            for (int b = 0; b < A::NK && b < nb && ok; ++b) ok = load_k(b);
+            for (int b = 0; b < nb && ok; ++b) {
+                ok = load_v(b);
+                if (ok && b + A::NK < nb) ok = load_k(b + A::NK);
             }
+            need_q();
         }
     } else if (warp == 1) {
         // ---------------- UMMA issuer ----------------
@@ -171,42 +203,38 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, KB);
             constexpr uint32_t idesc_pv = umma_idesc_bf16_bmn(128, 64);
             const uint64_t qd = umma_desc_k128(smem_u32(sQ));
+            const uint32_t sK = smem_u32(sKV), sV = sK + A::NK * A::KV_BYTES;
             bool ok = mbar_wait(q_full, 0, status);
-            auto issue_s = [&](int b) {          // S(b) = Q K(b)^T into group (b & 1)'s accumulator
-                const int s = b % A::NST, g = b & 1;
-                if (!mbar_wait(kv_full + 8 * s, (b / A::NST) & 1, status)) return false;
+            auto issue_s = [&](int b) {          // S(b) = Q K(b)^T into accumulator b % 3
+                const int st = b % A::NK;
+                if (!mbar_wait(k_full + 8 * st, (b / A::NK) & 1, status)) return false;
                 tc_fence_after();
-                const uint64_t kd = umma_desc_k128(smem_u32(sKV + s * 2 * A::KV_BYTES));
+                const uint64_t kd = umma_desc_k128(sK + st * A::KV_BYTES);
 #pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4) umma_bf16_ss(tmem + 128 * g, qd + 2 * k4, kd + 2 * k4, idesc_s, k4 != 0);
-                umma_commit(s_full + 8 * g);
+                for (int k4 = 0; k4 < 4; ++k4) umma_bf16_ss(tmem + 128 * st, qd + 2 * k4, kd + 2 * k4, idesc_s, k4 != 0);
+                umma_commit(s_full + 8 * st);    // S(b) is ready; K's stage is free
                 return true;
             };
-            // The two groups share each scheduler's special-function unit.  Started together they stay in step:
-            // both wait for their S at the same time and both exponentiate at the same time, at half the
-            // rate each.  Group 1's first S is therefore issued only when group 0 is half way through its
-            // first block, which puts the groups in opposite phases: one exponentiates while the other waits.
-            if (ok) ok = issue_s(0);
-            if (ok && nb > 1) ok = mbar_wait(stagger, 0, status) && issue_s(1);
+            for (int b = 0; b < A::NK && b < nb && ok; ++b) ok = issue_s(b);
             for (int b = 0; b < nb && ok; ++b) {
-                const int g = b & 1, s = b % A::NST;
-                ok = mbar_wait(p_full + 8 * g, (b >> 1) & 1, status);
+                const int g = b & 1, sv = b % A::NV;
+                ok = mbar_wait(p_full + 8 * g, (b >> 1) & 1, status) && mbar_wait(v_full + 8 * sv, (b / A::NV) & 1, status);
                 if (!ok) break;
-                // the group has consumed S(b): its next S goes first, so that it is ready as early as possible
-                if (b + 2 < nb) ok = issue_s(b + 2);
-                if (!ok) break;
+                if (b == 4) NFD_TRACE_MARK_T(TRK_OTHER + 6, 32);
                 tc_fence_after();
-                const uint64_t pd = umma_desc_k128(smem_u32(sP + g * A::P_BYTES));
-                const uint64_t vd = umma_desc_k128(smem_u32(sKV + s * 2 * A::KV_BYTES + A::KV_BYTES));
+                const uint64_t vd = umma_desc_k128(sV + sv * A::KV_BYTES);
+                const uint32_t tP = tmem + 128 * (b % A::NK);
 #pragma unroll
                 for (int i = 0; i < KB / 16; ++i) {
-                    // P: K-major, 64-key atoms of 16 KiB; V: MN-major, 16 keys = 2 KiB per step
-                    const uint64_t pa = pd + (uint64_t)((i >> 2) * (16384 >> 4) + (i & 3) * 2);
-                    umma_bf16_ss(tmem + 256 + 64 * g, pa, vd + (uint64_t)(i * (2048 >> 4)), idesc_pv,
+                    // P: 16 keys = 8 columns of packed bf16 pairs; V: MN-major, 16 keys = 2 KiB per step
+                    umma_bf16_ts(tmem + 384 + 64 * g, tP + 8 * i, vd + (uint64_t)(i * (2048 >> 4)), idesc_pv,
                                  (uint32_t)((b >> 1) != 0 || i != 0));
                 }
-                umma_commit(pv_done + 8 * g);
-                umma_commit(kv_empty + 8 * s);
+                umma_commit(v_empty + 8 * sv);   // P V(b) is complete: V's stage is free, the group's O at rest
+                if (b == 4) NFD_TRACE_MARK_T(TRK_OTHER + 7, 32);
+                // the group has read S(b): its accumulator takes the block three ahead
+                if (b + A::NK < nb) ok = issue_s(b + A::NK);
+                if (b == 4) NFD_TRACE_MARK_T(TRK_OTHER + 8, 32);
             }
         }
     } else {
@@ -215,14 +243,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
         const int quad = warp & 3;
         const int trow = quad * 32 + lane;
         const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
-        const uint32_t tS = tmem + 128 * g + lane_off, tO = tmem + 256 + 64 * g + lane_off;
+        const uint32_t tO = tmem + 384 + 64 * g + lane_off;
         const float c = (1.0f / sqrtf((float)D.dh)) * 1.4426950408889634f;   // softmax scale in the log2 domain
         float m_run = -INFINITY, l_run = 0.f;
-        uint8_t *prow = sP + g * A::P_BYTES + trow * 128;
         bool ok = true;
         int i = 0;
         for (int b = g; b < nb; b += 2, ++i) {
-            ok = mbar_wait(s_full + 8 * g, i & 1, status);
+            const uint32_t tS = tmem + 128 * (b % A::NK) + lane_off;
+            ok = mbar_wait(s_full + 8 * (b % A::NK), (b / A::NK) & 1, status);
             if (!ok) break;
             tc_fence_after();
             if (i == 0) NFD_TRACE_MARK_T(TRK_OTHER + 11, 64);
@@ -245,17 +273,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
             }
             const float m_blk = mx * c;
-            if (i > 0) {
-                // the previous P V product of this group is complete: its P tile is free, O is at rest
-                ok = mbar_wait(pv_done + 8 * g, (i - 1) & 1, status);
-                if (!ok) break;
-                tc_fence_after();
-            }
             const bool raise = m_blk > m_run + 8.0f;       // always true for the first block (m_run = -inf)
             if (__any_sync(0xffffffffu, raise)) {
                 const float m_new = raise ? m_blk : m_run;
                 const float f = ex2_approx(m_run - m_new);  // 1 for rows that keep their reference maximum
                 if (i > 0) {
+                    // the previous P V product of this group must be complete before O is touched
+                    ok = mbar_wait(v_empty + 8 * ((b - 2) % A::NV), ((b - 2) / A::NV) & 1, status);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
                     for (int cc = 0; cc < 64; cc += 32) {
                         uint32_t r[32];
@@ -270,8 +296,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 l_run *= f;
                 m_run = m_new;
             }
-            // pass 2 over S, 16 columns at a time with the next load in flight:
-            // P = exp2(S c - m) as bf16 into shared memory (128-byte-swizzled K-major layout)
+            // pass 2 over S, 16 columns at a time with the next load in flight: P = exp2(S c - m) as packed bf16
+            // pairs, written over the columns of S that have been read already (keys k .. k+15 go to columns
+            // k/2 .. k/2+7, which never reach ahead of the columns still to be read)
             float2 ls2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
             uint32_t sa[16], sb[16];
             tmem_ld16(tS, sa);
@@ -280,27 +307,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
                 uint32_t *cur = ((cc >> 4) & 1) ? sb : sa, *nxt = ((cc >> 4) & 1) ? sa : sb;
                 tmem_ld_wait();
                 if (cc + 16 < KB) tmem_ld16(tS + cc + 16, nxt);
-                if (cc == (KB / 32) * 16 && g == 0 && i == 0) mbar_arrive(stagger);     // see the UMMA issuer
+                uint32_t pk[8];
 #pragma unroll
-                for (int u2 = 0; u2 < 2; ++u2) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float2 y = ffma2(make_float2(__uint_as_float(cur[8 * u2 + 2 * u]),
-                                                           __uint_as_float(cur[8 * u2 + 2 * u + 1])),
-                                               make_float2(c, c), make_float2(-m_run, -m_run));
-                        const float p0 = ex2_approx(y.x), p1 = ex2_approx(y.y);
-                        ls2[u] = fadd2(ls2[u], make_float2(p0, p1));
-                        const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
-                        pk[u] = *reinterpret_cast<const uint32_t *>(&hp);
-                    }
-                    const int ch = (cc >> 3) + u2;
-                    uint8_t *dst = prow + (ch >> 3) * 16384 + (((ch & 7) ^ (trow & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                for (int u = 0; u < 8; ++u) {
+                    const float2 y = ffma2(make_float2(__uint_as_float(cur[2 * u]), __uint_as_float(cur[2 * u + 1])),
+                                           make_float2(c, c), make_float2(-m_run, -m_run));
+                    const float p0 = ex2_approx(y.x), p1 = ex2_approx(y.y);
+                    ls2[u & 3] = fadd2(ls2[u & 3], make_float2(p0, p1));
+                    const __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
+                    pk[u] = *reinterpret_cast<const uint32_t *>(&hp);
                 }
+                tmem_st8(tS + (cc >> 1), pk);
             }
             l_run += ((ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y)) + ((ls2[2].x + ls2[2].y) + (ls2[3].x + ls2[3].y));
-            fence_proxy_async_smem();
+            tmem_st_wait();                                // P is in tensor memory
             tc_fence_before();
             mbar_arrive(p_full + 8 * g);
         }
@@ -310,7 +330,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUten
 #pragma unroll
         for (int e = 0; e < 64; ++e) O[e] = 0.f;
         if (ok && i > 0) {
-            ok = mbar_wait(pv_done + 8 * g, (i - 1) & 1, status);
+            const int bl = g + 2 * (i - 1);                  // this group's last block
+            ok = mbar_wait(v_empty + 8 * (bl % A::NV), (bl / A::NV) & 1, status);
             if (ok) {
                 tc_fence_after();
 #pragma unroll
