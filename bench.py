@@ -302,7 +302,7 @@ def profile_case(argv):
     """Small, self-ending workload for profiler captures of the library's kernels:
 
         python bench.py --profile-case [--layers 2] [--ctx 16] [--k 1] [--passes 2] [--no-graph] [--no-fast]
-                                       [--no-prefetch]
+                                       [--no-prefetch] [--kv-prefetch] [--time N]
 
     The 310M-class shape with few layers (well under a GB on the device), the KV context filled by commit
     passes, then a few denoising passes.  Meant to be wrapped by `ncu -k regex:... -c N`."""
@@ -317,7 +317,11 @@ def profile_case(argv):
     ap.add_argument("--passes", type=int, default=2)
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--no-prefetch", action="store_true")
+    ap.add_argument("--no-prefetch", action="store_true", help="GEMMs do not pull the next GEMM's weights towards L2")
+    ap.add_argument("--kv-prefetch", action="store_true",
+                    help="the QKV GEMM pulls the layer's cached K/V pages towards L2 (off by default)")
+    ap.add_argument("--time", type=int, default=0, metavar="N",
+                    help="also time N passes between two CUDA events (graph replay) and print microseconds per pass")
     a = ap.parse_args(argv)
     cfg = I.make_cfg("nfd310m", n_layers=a.layers, ctx_frames=a.ctx)
     dev = torch.device("cuda:0")
@@ -328,6 +332,8 @@ def profile_case(argv):
         nfd.set_option("fast", 0)
     if a.no_prefetch:
         nfd.set_option("l2_prefetch", 0)
+    if a.kv_prefetch:
+        nfd.set_option("kv_prefetch", 1)
     g = torch.Generator(device=dev)
     g.manual_seed(0)
     fs = I.frame_shape(cfg)
@@ -338,6 +344,20 @@ def profile_case(argv):
     for _ in range(a.passes):
         v = nfd.denoise_step(x, 0.7, 3)
     torch.cuda.synchronize()
+    if a.time > 0:
+        best = None
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(nfd.stream):
+                e0.record(nfd.stream)
+                for _ in range(a.time):
+                    nfd.denoise_step(x, 0.7, 3)
+                e1.record(nfd.stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / a.time
+            best = us if best is None else min(best, us)
+        print(f"layers={a.layers} k={a.k} kv_prefetch={int(a.kv_prefetch)} weight_prefetch={int(not a.no_prefetch)}: "
+              f"{best:.1f} us per pass ({best / a.layers:.2f} per layer), best of 3 x {a.time} passes")
     assert nfd.status() == 0
     print("ok", float(v.abs().mean()))
     return 0

@@ -302,9 +302,10 @@ int nfd_warm_modulation(nfd_ctx *ctx);
  * once), "fuse_ln" 0/1 (bf16 tensor-core path: fold the two adaLN LayerNorms of
  * every block into the epilogues of the neighbouring GEMMs, or run them as
  * kernels of their own; the two differ by bf16 rounding of the GEMM operand
- * only), "l2_prefetch" 0/1 (each GEMM pulls the next GEMM's weights, the QKV
- * GEMM also the layer's cached K/V pages, towards L2), "clear_status" (reset the
- * device-side status latch).  Changing "fast" or "fuse_ln" empties the
+ * only), "l2_prefetch" 0/1 (each GEMM pulls the next GEMM's weights towards
+ * L2; on by default), "kv_prefetch" 0/1 (the QKV GEMM pulls the layer's cached
+ * K/V pages towards L2 ahead of the attention kernel; off by default, it was
+ * measured slower), "clear_status" (reset the device-side status latch).  Changing "fast" or "fuse_ln" empties the
  * modulation cache.
  * Switches that exist for the tests of the error paths; each makes a fault on
  * the host or lets a bounded wait expire, none makes the device fault:
