@@ -302,7 +302,7 @@ def profile_case(argv):
     """Small, self-ending workload for profiler captures of the library's kernels:
 
         python bench.py --profile-case [--layers 2] [--ctx 16] [--k 1] [--passes 2] [--no-graph] [--no-fast]
-                                       [--no-prefetch] [--kv-prefetch] [--time N]
+                                       [--no-prefetch] [--kv-prefetch] [--streams 8] [--time N]
 
     The 310M-class shape with few layers (well under a GB on the device), the KV context filled by commit
     passes, then a few denoising passes.  Meant to be wrapped by `ncu -k regex:... -c N`."""
@@ -320,10 +320,12 @@ def profile_case(argv):
     ap.add_argument("--no-prefetch", action="store_true", help="GEMMs do not pull the next GEMM's weights towards L2")
     ap.add_argument("--kv-prefetch", action="store_true",
                     help="the QKV GEMM pulls the layer's cached K/V pages towards L2 (off by default)")
+    ap.add_argument("--streams", type=int, default=1,
+                    help="independent streams, each with its own context; the denoising passes are batched over them")
     ap.add_argument("--time", type=int, default=0, metavar="N",
                     help="also time N passes between two CUDA events (graph replay) and print microseconds per pass")
     a = ap.parse_args(argv)
-    cfg = I.make_cfg("nfd310m", n_layers=a.layers, ctx_frames=a.ctx)
+    cfg = I.make_cfg("nfd310m", n_layers=a.layers, ctx_frames=a.ctx, n_streams=a.streams)
     dev = torch.device("cuda:0")
     nfd = NFD(cfg, torch_weights(cfg, dev, seed=0))
     if a.no_graph:
@@ -337,12 +339,19 @@ def profile_case(argv):
     g = torch.Generator(device=dev)
     g.manual_seed(0)
     fs = I.frame_shape(cfg)
-    for i in range(0, a.ctx, 4):
-        n = min(4, a.ctx - i)
-        nfd.commit_frame(torch.randn((n,) + fs, generator=g, device=dev), [1] * n)
-    x = torch.randn((a.k,) + fs, generator=g, device=dev)
+    streams = list(range(a.streams))
+    for st in streams:
+        for i in range(0, a.ctx, 4):
+            n = min(4, a.ctx - i)
+            nfd.commit_frame(torch.randn((n,) + fs, generator=g, device=dev), [1] * n, stream=st)
+    if a.streams == 1:
+        x = torch.randn((a.k,) + fs, generator=g, device=dev)
+        step = lambda: nfd.denoise_step(x, 0.7, 3)
+    else:
+        x = torch.randn((a.streams, a.k) + fs, generator=g, device=dev)
+        step = lambda: nfd.denoise_step_batched(streams, x, [0.7] * a.streams, [3] * a.streams)
     for _ in range(a.passes):
-        v = nfd.denoise_step(x, 0.7, 3)
+        v = step()
     torch.cuda.synchronize()
     if a.time > 0:
         best = None
@@ -351,7 +360,7 @@ def profile_case(argv):
             with torch.cuda.stream(nfd.stream):
                 e0.record(nfd.stream)
                 for _ in range(a.time):
-                    nfd.denoise_step(x, 0.7, 3)
+                    step()
                 e1.record(nfd.stream)
             torch.cuda.synchronize()
             us = e0.elapsed_time(e1) * 1e3 / a.time
@@ -706,7 +715,7 @@ def main():
             b8 = {"aggregate_frames_per_s": round(nb * n8 / (ms8 * 1e-3), 2),
                   "per_stream_frames_per_s": round(n8 / (ms8 * 1e-3), 2),
                   "ms_per_batched_frame_step": round(ms8 / n8, 3), "streams": nb, "ctx_frames": 32, "steps": n8,
-                  "workload": "BASELINE config 5: 8 independent streams, 32-frame KV context, 4 steps + commit"}
+                  "workload": "8 independent streams, 32-frame KV context each, 4 steps + commit, one batched call per frame"}
             # its dominant kernel: teacher-forced batched passes of 8 x 1 frames behind the full contexts
             fill8()
             xt8 = randn(nb, 1, *fs)

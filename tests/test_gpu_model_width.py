@@ -30,7 +30,7 @@ def _kv_check(g, orc, layers, frames, what, stream=0, scale=False):
 
 
 def test_four_frame_pass_and_speculation_at_model_width():
-    """Config 4's pass: k = 4 frames (1344 query rows, block-causal among themselves) on a two-layer slice with
+    """Four speculative frames in one pass: k = 4 frames (1344 query rows, block-causal among themselves) on a two-layer slice with
     the stress weights.  First one teacher-forced pass (velocity and the K/V pages it leaves), then a full
     speculation of four frames with two of them accepted, against the oracle doing the same."""
     cfg = I.make_cfg("nfd310m_slice")
@@ -62,7 +62,7 @@ def test_four_frame_pass_and_speculation_at_model_width():
 
 
 def test_batched_streams_behind_a_full_32_frame_context():
-    """Config 5's structure on a two-layer slice: a context made for 8 streams with a 32-frame window.  Three
+    """Batched streams on a two-layer slice: a context made for 8 streams with a 32-frame window.  Three
     of the streams get 34, 37 and 42 committed frames (window full, oldest frames evicted, the last one past
     the ring's wrap-around), then one batched speculation; each stream against an oracle of its own."""
     from paper_2506_01380_b200.nfd import NFD
@@ -123,7 +123,7 @@ def test_free_running_six_layers_stress_weights():
 
 
 def test_free_running_full_depth():
-    """The same on all 24 layers of config 3, with the N(0, 0.02^2) weights the configuration names."""
+    """The same on all 24 layers of the 310M-class model, with N(0, 0.02^2) weights."""
     _free_running(I.make_cfg("nfd310m"), "paper", seed=4, n_prompt=16, n_gen=4)
 
 

@@ -87,7 +87,7 @@ CASES = [
 
 @pytest.mark.parametrize("name,kind,opts", CASES)
 def test_denoise_step_after_prompt(name, kind, opts):
-    """Config 1: 4 prompt frames in the cache, one denoising step for one new frame."""
+    """The tiny model: 4 prompt frames in the cache, one denoising step for one new frame."""
     cfg = I.make_cfg(name)
     g, orc = make_pair(cfg, 0, kind, **opts)
     acts = prompt(cfg, g, orc, 4, seed=100, group=2)
@@ -276,7 +276,7 @@ def test_error_codes_leave_state_unchanged():
 @pytest.mark.parametrize("fast", [0, 1])
 @pytest.mark.parametrize("n_kv,n_q,window", [(5, 1, 64), (17, 1, 64), (65, 1, 64), (17, 4, 16), (9, 3, 2)])
 def test_attention_alone(n_kv, n_q, window, fast):
-    """Config 2: 16 heads x 64, 336-token frames, block-causal over the cache."""
+    """Attention alone: 16 heads x 64, 336-token frames, block-causal over the cache."""
     torch = _torch()
     from paper_2506_01380_b200.nfd import NFD
     cfg = I.make_cfg("nfd310m", n_layers=1, ctx_frames=64, max_spec=4)
@@ -333,7 +333,7 @@ def test_paper_130m_and_774m_shapes_one_layer():
 
 
 def test_310m_full_config_teacher_forced():
-    """Config 3's shape: 24 layers, 16 context frames, one denoising pass, GPU vs oracle."""
+    """The 310M-class shape: 24 layers, 16 context frames, one denoising pass, GPU vs oracle."""
     _teacher_forced(I.make_cfg("nfd310m"), "paper", n_prompt=16, k=1, seed=0)
 
 
@@ -468,7 +468,7 @@ def test_deferred_commit_equals_immediate_commit(name):
 
 
 def test_batch8_streams_at_model_width_match_single_streams():
-    """Config 5's structure (8 independent streams, 32-frame context) on a 2-layer slice of the 310M-class
+    """Batched decoding (8 independent streams, 32-frame context) on a 2-layer slice of the 310M-class
     width: one batched speculation must give bitwise the frames and caches of eight single-stream ones."""
     from paper_2506_01380_b200.nfd import NFD
     torch = _torch()
